@@ -1,0 +1,186 @@
+/*
+ * vt.h - C boundary of the trimmed-vocabulary draft head for NVIDIA B200 (sm_100a).
+ *
+ * The library computes, on one GPU, the part of a speculative-decoding draft step that
+ * vocabulary trimming makes cheaper: the draft model's language-modelling head restricted to
+ * a kept set V_d of V_trim token rows (the paper's k = |V_d|, Section 2.1), whose cost is the
+ * 2*d*k term of the paper's cost model (Section 2.3, Eq. 3).
+ *
+ * Conventions that hold for every entry point
+ *  - "dev" pointers are device memory of the current CUDA device, "host" pointers are host
+ *    memory.  The caller owns every buffer; the library allocates and frees nothing and keeps
+ *    no pointer after a call returns.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Unless stated
+ *    otherwise a call only enqueues work on that stream and returns without synchronising.
+ *  - bf16 tensors are row-major arrays of 16-bit patterns; ids and indices are int32.
+ *  - Errors are return codes.  Argument errors are detected on the host before anything is
+ *    launched.  No entry point throws, aborts or traps the device.
+ *  - A call must run on the device whose memory it is given; the library does not switch devices.
+ */
+#ifndef VT_H_
+#define VT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum vt_status {
+    VT_OK = 0,
+    VT_ERR_NULL = 1,       /* a required pointer is NULL                                              */
+    VT_ERR_SHAPE = 2,      /* d < 8, d % 8 != 0, M < 1, V_trim < 1, V_trim > V_full, k < 1, k > V_trim,
+                              k > VT_MAX_K, N < 0, a size beyond what an entry point states it takes  */
+    VT_ERR_ALIGN = 3,      /* a bf16 matrix pointer is not 16-byte aligned, an id pointer not 4-byte  */
+    VT_ERR_RANGE = 4,      /* a keep id lies outside [0, V_full)                                      */
+    VT_ERR_DUP = 5,        /* keep_ids names an id twice (V_d is a set, Section 2.1)                  */
+    VT_ERR_EMPTY = 6,      /* vt_coverage with N == 0: Eq. 2 would be 0/0                             */
+    VT_ERR_WORKSPACE = 7,  /* workspace NULL, misaligned (256 B) or smaller than the size function says */
+    VT_ERR_TIMEOUT = 8,    /* a bounded device-side wait ran out; outputs of that call are invalid    */
+    VT_ERR_CUDA = 9,       /* a CUDA runtime or driver call failed (see vt_last_cuda_error)           */
+    VT_ERR_UNSUPPORTED = 10 /* the requested path cannot run this shape (only with a forced path)     */
+} vt_status;
+
+#define VT_MAX_K 64        /* largest top-k per draft row */
+
+/* Which contraction kernel vt_draft_head_path / vt_debug_logits run. */
+typedef enum vt_path {
+    VT_PATH_AUTO = 0,      /* chosen from M and d                                                     */
+    VT_PATH_GEMV = 1,      /* CUDA-core streaming GEMV; M <= 8 per pass and d <= 8192                 */
+    VT_PATH_MMA = 2        /* tcgen05 tensor-core GEMM with TMEM accumulators; any M                   */
+} vt_path;
+
+/* Text for a status code (static storage). */
+const char* vt_strerror(vt_status s);
+
+/* The last CUDA error code (cudaError_t or CUresult as int) this thread's calls ran into; 0 if none. */
+int vt_last_cuda_error(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Head compaction (Section 2.1: the draft vocabulary V_d is the kept tokens; the head keeps
+ * only their rows).
+ *
+ *   W_trim[i, :] = W_full[keep_ids[i], :]      for i in [0, V_trim),  a bit copy of bf16 rows
+ *
+ *   W_full   dev  [V_full, d] bf16 row-major, 16-byte aligned
+ *   keep_ids dev  [V_trim] int32, each in [0, V_full), pairwise distinct (not checked here:
+ *                 vt_validate_keep_ids does that; an out-of-range id is skipped and sets
+ *                 VT_ERR_RANGE in no status word - validate first)
+ *   W_trim   dev  [V_trim, d] bf16 row-major, caller-allocated, 16-byte aligned, must not
+ *                 overlap W_full
+ * Asynchronous.  VT_ERR_NULL / VT_ERR_SHAPE / VT_ERR_ALIGN / VT_ERR_CUDA.
+ */
+vt_status vt_compact_head(const void* W_full, int V_full, int d,
+                          const int32_t* keep_ids, int V_trim,
+                          void* W_trim, void* stream);
+
+/* Bytes of scratch vt_validate_keep_ids and vt_coverage need for a vocabulary of V_full ids
+ * (a membership bitmap plus counters).  Returns 0 if V_full < 1. */
+size_t vt_coverage_workspace_bytes(int V_full);
+
+/* Checks that keep_ids is a set inside [0, V_full) (Section 2.1).  Builds the membership
+ * bitmap in `workspace` (dev, 256-byte aligned, vt_coverage_workspace_bytes(V_full)) and
+ * SYNCHRONISES the stream to read two counters back.
+ * Returns VT_ERR_RANGE if any id is out of range, else VT_ERR_DUP if any id repeats, else VT_OK. */
+vt_status vt_validate_keep_ids(const int32_t* keep_ids, int V_trim, int V_full,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Draft head over the trimmed vocabulary (Section 2.3: the d -> k linear head, the only
+ * vocabulary-dependent cost of an EAGLE-style draft; Section 1: the draft-to-target buffer).
+ *
+ * For each draft row m in [0, M):
+ *   x[m, i]   = sum_j h[m, j] * W_trim[i, j]            fp32 accumulation of exact bf16 products
+ *   lse[m]    = log sum_{i < V_trim} exp(x[m, i])       natural log, over the kept rows only
+ *   the k largest x[m, :] in descending order, equal logits ordered by ascending draft index
+ *   logprobs[m, j]   = x[m, i_j] - lse[m]
+ *   target_ids[m, j] = d2t[i_j]                         d2t holds absolute target-vocabulary ids
+ * The logits are never written to memory.
+ *
+ *   h          dev [M, d] bf16, 16-byte aligned          W_trim dev [V_trim, d] bf16, 16-byte aligned
+ *   d2t        dev [V_trim] int32
+ *   target_ids dev [M, k] int32 (out)                    logprobs dev [M, k] float (out)
+ *   draft_ids  dev [M, k] int32 (out) or NULL            lse      dev [M] float (out) or NULL
+ *   workspace  dev, 256-byte aligned, at least vt_workspace_bytes(M, k) bytes, zero-filled once
+ *              by vt_workspace_init before its first use.  It carries per-CTA partial results,
+ *              an arrival counter and a status word; calls that share a workspace must be
+ *              ordered on one stream.
+ * d % 8 == 0, d >= 8; 1 <= k <= min(V_trim, VT_MAX_K); any M >= 1.  Inputs must be finite.
+ * Asynchronous: no host synchronisation.  A device-side wait that ran out is reported by
+ * vt_last_status on the same workspace.
+ */
+size_t    vt_workspace_bytes(int M, int k);
+vt_status vt_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+vt_status vt_draft_head(const void* h, const void* W_trim, const int32_t* d2t,
+                        int M, int d, int V_trim, int k,
+                        int32_t* target_ids, float* logprobs,
+                        int32_t* draft_ids, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same call with the contraction kernel forced (VT_ERR_UNSUPPORTED if that kernel cannot take
+ * the shape).  VT_PATH_AUTO is what vt_draft_head uses. */
+vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d2t,
+                             int M, int d, int V_trim, int k,
+                             int32_t* target_ids, float* logprobs,
+                             int32_t* draft_ids, float* lse,
+                             void* workspace, size_t workspace_bytes, void* stream, int path);
+
+/* End-to-end form of vt_draft_head for callers whose per-step data lives on the host:
+ * h_host (host [M, d] bf16, ideally pinned) is copied to the device, the head runs, and
+ * target_ids_host / logprobs_host (host [M, k]) are copied back, all on `stream`; the call
+ * SYNCHRONISES the stream before returning so the host outputs are valid.  W_trim and d2t
+ * stay device-resident (they are model state, not per-step input).
+ * workspace: dev, vt_host_workspace_bytes(M, d, k) bytes, initialised with vt_workspace_init. */
+size_t    vt_host_workspace_bytes(int M, int d, int k);
+vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32_t* d2t,
+                             int M, int d, int V_trim, int k,
+                             int32_t* target_ids_host, float* logprobs_host,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Reads the status word of a draft-head workspace.  SYNCHRONISES the stream.  Returns VT_OK,
+ * VT_ERR_TIMEOUT, or VT_ERR_CUDA, and clears the word. */
+vt_status vt_last_status(void* workspace, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Coverage of a token stream by the kept set (Eq. 2 with f(v) = occurrences of v in the
+ * stream; the "frequency coverage" of Table 4):
+ *
+ *   covered = #{ t in [0, N) : token_ids[t] in keep_ids },   fraction = covered / N
+ *
+ *   token_ids dev [N] int32; ids outside [0, V_full) count in N and are never covered
+ *   keep_ids  dev [V_trim] int32 in [0, V_full) (out-of-range entries are ignored)
+ *   covered_out, fraction_out: host (either may be NULL)
+ *   workspace dev, 256-byte aligned, vt_coverage_workspace_bytes(V_full) bytes; contents are
+ *             overwritten, no initialisation needed
+ * SYNCHRONISES the stream once to return the count.  N == 0 gives VT_ERR_EMPTY.
+ */
+vt_status vt_coverage(const int32_t* token_ids, int64_t N,
+                      const int32_t* keep_ids, int V_trim, int V_full,
+                      uint64_t* covered_out, double* fraction_out,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Test and inspection entry points (same kernels as the calls above).
+ */
+
+/* The head contraction alone (Section 2.3), with the epilogue storing x[m, i] as fp32:
+ * logits dev [M, V_trim] row-major (out).  Runs the same contraction code as vt_draft_head
+ * on the chosen path; workspace as for vt_draft_head with k = 1. */
+vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V_trim,
+                          float* logits, void* workspace, size_t workspace_bytes,
+                          void* stream, int path);
+
+/* The draft-to-target map alone (Section 1): target_ids[t] = d2t[draft_ids[t]] for t < n.
+ * A draft id outside [0, V_trim) writes -1.  All pointers dev. */
+vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
+                   int32_t* target_ids, void* stream);
+
+/* Number of kernels the last call of this thread launched (for launch accounting). */
+int vt_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VT_H_ */

@@ -1,0 +1,223 @@
+"""Python binding of ``libvt.so``: argument marshalling only.
+
+Each function has the name of the C entry point it calls (``include/vt.h``) and passes torch
+tensors' device pointers and the current CUDA stream through ctypes.  PyTorch provides device
+memory and streams; every step of the head runs inside the library's kernels.  There is no
+fallback: if the library cannot be loaded the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvt.so")
+
+VT_OK = 0
+VT_ERR_NULL, VT_ERR_SHAPE, VT_ERR_ALIGN, VT_ERR_RANGE, VT_ERR_DUP = 1, 2, 3, 4, 5
+VT_ERR_EMPTY, VT_ERR_WORKSPACE, VT_ERR_TIMEOUT, VT_ERR_CUDA, VT_ERR_UNSUPPORTED = 6, 7, 8, 9, 10
+VT_MAX_K = 64
+VT_PATH_AUTO, VT_PATH_GEMV, VT_PATH_MMA = 0, 1, 2
+
+# every symbol include/vt.h declares: name -> (restype, argtypes)
+_p, _i, _i64, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+SYMBOLS = {
+    "vt_strerror": (ctypes.c_char_p, [_i]),
+    "vt_last_cuda_error": (_i, []),
+    "vt_compact_head": (_i, [_p, _i, _i, _p, _i, _p, _p]),
+    "vt_coverage_workspace_bytes": (_sz, [_i]),
+    "vt_validate_keep_ids": (_i, [_p, _i, _i, _p, _sz, _p]),
+    "vt_workspace_bytes": (_sz, [_i, _i]),
+    "vt_workspace_init": (_i, [_p, _sz, _p]),
+    "vt_draft_head": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _p, _p, _sz, _p]),
+    "vt_draft_head_path": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _p, _p, _sz, _p, _i]),
+    "vt_host_workspace_bytes": (_sz, [_i, _i, _i]),
+    "vt_draft_head_host": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _sz, _p]),
+    "vt_last_status": (_i, [_p, _p]),
+    "vt_coverage": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p, _sz, _p]),
+    "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
+    "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
+    "vt_last_launch_count": (_i, []),
+}
+
+_lib = None
+
+
+class VtError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = int(status)
+        text = lib().vt_strerror(self.status).decode()
+        extra = f" (CUDA error {lib().vt_last_cuda_error()})" if self.status == VT_ERR_CUDA else ""
+        super().__init__(f"{what}: status {self.status}: {text}{extra}")
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libvt.so`` from the package directory, building it with nvcc first if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            from .build import build
+            build()
+        cd = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(cd, name)     # AttributeError if the library lacks a declared symbol
+            fn.restype, fn.argtypes = res, args
+        _lib = cd
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != VT_OK:
+        raise VtError(status, what)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _bf16(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.dtype not in (torch.bfloat16, torch.int16, torch.uint16):
+        raise TypeError(f"{name}: expected bf16 data (torch.bfloat16 or a 16-bit integer view), got {t.dtype}")
+    if not t.is_cuda or not t.is_contiguous() or t.dim() != 2:
+        raise ValueError(f"{name}: expected a contiguous 2-D CUDA tensor")
+    return t
+
+
+def _i32(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name}: expected a contiguous int32 CUDA tensor")
+    return t
+
+
+def vt_workspace_bytes(M: int, k: int) -> int:
+    return int(lib().vt_workspace_bytes(M, k))
+
+
+def vt_host_workspace_bytes(M: int, d: int, k: int) -> int:
+    return int(lib().vt_host_workspace_bytes(M, d, k))
+
+
+def vt_coverage_workspace_bytes(V_full: int) -> int:
+    return int(lib().vt_coverage_workspace_bytes(V_full))
+
+
+def vt_workspace_init(workspace: torch.Tensor) -> torch.Tensor:
+    _check(lib().vt_workspace_init(workspace.data_ptr(), workspace.numel(), _stream()), "vt_workspace_init")
+    return workspace
+
+
+def new_workspace(nbytes: int, device=None) -> torch.Tensor:
+    """A zero-initialised byte buffer of the caller's (torch's caching allocator is 512-byte aligned)."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device or "cuda")
+    return vt_workspace_init(ws)
+
+
+def vt_compact_head(W_full: torch.Tensor, keep_ids: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    W_full = _bf16(W_full, "W_full")
+    keep_ids = _i32(keep_ids, "keep_ids")
+    V, d = W_full.shape
+    Vt = keep_ids.numel()
+    if out is None:
+        out = torch.empty((Vt, d), dtype=W_full.dtype, device=W_full.device)
+    _check(lib().vt_compact_head(W_full.data_ptr(), V, d, keep_ids.data_ptr(), Vt, out.data_ptr(), _stream()),
+           "vt_compact_head")
+    return out
+
+
+def vt_validate_keep_ids(keep_ids: torch.Tensor, V_full: int, workspace: torch.Tensor | None = None) -> int:
+    """Returns the status (VT_OK, VT_ERR_RANGE or VT_ERR_DUP) instead of raising for those two."""
+    keep_ids = _i32(keep_ids, "keep_ids")
+    if workspace is None:
+        workspace = torch.empty(vt_coverage_workspace_bytes(V_full), dtype=torch.uint8, device=keep_ids.device)
+    st = lib().vt_validate_keep_ids(keep_ids.data_ptr(), keep_ids.numel(), V_full, workspace.data_ptr(),
+                                    workspace.numel(), _stream())
+    if st not in (VT_OK, VT_ERR_RANGE, VT_ERR_DUP):
+        raise VtError(st, "vt_validate_keep_ids")
+    return st
+
+
+def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, d2t: torch.Tensor, k: int, *,
+                  workspace: torch.Tensor | None = None, path: int = VT_PATH_AUTO,
+                  target_ids: torch.Tensor | None = None, logprobs: torch.Tensor | None = None,
+                  draft_ids: torch.Tensor | None = None, lse: torch.Tensor | None = None):
+    """(target_ids [M,k] int32, logprobs [M,k] float32); pass ``draft_ids`` / ``lse`` tensors to receive those too."""
+    h = _bf16(h, "h")
+    W_trim = _bf16(W_trim, "W_trim")
+    d2t = _i32(d2t, "d2t")
+    M, d = h.shape
+    Vt, d2 = W_trim.shape
+    if d2 != d or d2t.numel() != Vt:
+        raise ValueError("h, W_trim and d2t disagree on d or V_trim")
+    if workspace is None:
+        workspace = new_workspace(vt_workspace_bytes(M, min(max(k, 1), VT_MAX_K)), h.device)
+    if target_ids is None:
+        target_ids = torch.empty((M, k), dtype=torch.int32, device=h.device)
+    if logprobs is None:
+        logprobs = torch.empty((M, k), dtype=torch.float32, device=h.device)
+    _check(lib().vt_draft_head_path(h.data_ptr(), W_trim.data_ptr(), d2t.data_ptr(), M, d, Vt, k,
+                                    target_ids.data_ptr(), logprobs.data_ptr(), _ptr(draft_ids), _ptr(lse),
+                                    workspace.data_ptr(), workspace.numel(), _stream(), path), "vt_draft_head")
+    return target_ids, logprobs
+
+
+def vt_draft_head_host(h_host: torch.Tensor, W_trim: torch.Tensor, d2t: torch.Tensor, k: int,
+                       target_ids_host: torch.Tensor, logprobs_host: torch.Tensor, workspace: torch.Tensor):
+    """Host-buffer form: ``h_host`` and both outputs are CPU tensors (pinned for speed); synchronises."""
+    M, d = h_host.shape
+    Vt = W_trim.shape[0]
+    if h_host.is_cuda or target_ids_host.is_cuda or logprobs_host.is_cuda:
+        raise ValueError("vt_draft_head_host takes host tensors for h and the outputs")
+    _check(lib().vt_draft_head_host(h_host.data_ptr(), W_trim.data_ptr(), d2t.data_ptr(), M, d, Vt, k,
+                                    target_ids_host.data_ptr(), logprobs_host.data_ptr(),
+                                    workspace.data_ptr(), workspace.numel(), _stream()), "vt_draft_head_host")
+    return target_ids_host, logprobs_host
+
+
+def vt_last_status(workspace: torch.Tensor) -> int:
+    return int(lib().vt_last_status(workspace.data_ptr(), _stream()))
+
+
+def vt_coverage(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int,
+                workspace: torch.Tensor | None = None) -> tuple[int, float]:
+    token_ids = _i32(token_ids, "token_ids")
+    keep_ids = _i32(keep_ids, "keep_ids")
+    if workspace is None:
+        workspace = torch.empty(vt_coverage_workspace_bytes(V_full), dtype=torch.uint8, device=keep_ids.device)
+    covered = ctypes.c_uint64(0)
+    frac = ctypes.c_double(0.0)
+    _check(lib().vt_coverage(token_ids.data_ptr() if token_ids.numel() else None, token_ids.numel(),
+                             keep_ids.data_ptr(), keep_ids.numel(), V_full,
+                             ctypes.addressof(covered), ctypes.addressof(frac),
+                             workspace.data_ptr(), workspace.numel(), _stream()), "vt_coverage")
+    return int(covered.value), float(frac.value)
+
+
+def vt_debug_logits(h: torch.Tensor, W_trim: torch.Tensor, path: int = VT_PATH_AUTO) -> torch.Tensor:
+    h = _bf16(h, "h")
+    W_trim = _bf16(W_trim, "W_trim")
+    M, d = h.shape
+    Vt = W_trim.shape[0]
+    logits = torch.empty((M, Vt), dtype=torch.float32, device=h.device)
+    ws = new_workspace(vt_workspace_bytes(M, 2), h.device)
+    _check(lib().vt_debug_logits(h.data_ptr(), W_trim.data_ptr(), M, d, Vt, logits.data_ptr(), ws.data_ptr(),
+                                 ws.numel(), _stream(), path), "vt_debug_logits")
+    return logits
+
+
+def vt_remap(draft_ids: torch.Tensor, d2t: torch.Tensor) -> torch.Tensor:
+    draft_ids = _i32(draft_ids, "draft_ids")
+    d2t = _i32(d2t, "d2t")
+    out = torch.empty_like(draft_ids)
+    _check(lib().vt_remap(draft_ids.data_ptr(), d2t.data_ptr(), draft_ids.numel(), d2t.numel(), out.data_ptr(),
+                          _stream()), "vt_remap")
+    return out
+
+
+def vt_last_launch_count() -> int:
+    return int(lib().vt_last_launch_count())

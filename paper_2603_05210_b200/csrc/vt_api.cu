@@ -1,0 +1,283 @@
+// C entry points: argument checks on the host, path choice, launches.  See include/vt.h for the contract.
+#include <cstdio>
+#include <cstring>
+
+#include "vt_launch.h"
+
+namespace vt {
+
+static thread_local int g_last_cuda_error = 0;
+static thread_local int g_launches = 0;
+
+vt_status cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return VT_ERR_CUDA;
+}
+vt_status driver_fail(int cu_result) {
+    g_last_cuda_error = cu_result;
+    return VT_ERR_CUDA;
+}
+void count_launch() { ++g_launches; }
+
+vt_status device_sm_count(int* sms) {
+    static int cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+    if (cached[dev] == 0) {
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        cached[dev] = n;
+    }
+    *sms = cached[dev];
+    return VT_OK;
+}
+
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+static vt_status check_head_args(const void* h, const void* W, const int32_t* d2t, int M, int d, int Vt, int k,
+                                 const void* target_ids, const void* logprobs, const void* ws, size_t ws_bytes) {
+    if (!h || !W || !d2t || !target_ids || !logprobs) return VT_ERR_NULL;
+    if (d < 8 || d % 8 != 0 || M < 1 || Vt < 1 || k < 1 || k > Vt || k > VT_MAX_K) return VT_ERR_SHAPE;
+    if (!aligned(h, 16) || !aligned(W, 16) || !aligned(d2t, 4) || !aligned(target_ids, 4) || !aligned(logprobs, 4))
+        return VT_ERR_ALIGN;
+    if (!ws || !aligned(ws, 256) || ws_bytes < ws_total_bytes(M, k)) return VT_ERR_WORKSPACE;
+    return VT_OK;
+}
+
+static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, float* lp, int32_t* did, float* lse,
+                        float* logits, void* ws) {
+    HeadOut o{};
+    o.d2t = d2t;
+    o.target_ids = tid;
+    o.logprobs = lp;
+    o.draft_ids = did;
+    o.lse = lse;
+    o.logits = logits;
+    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+    o.hdr = reinterpret_cast<WsHeader*>(base);
+    o.keys = reinterpret_cast<unsigned long long*>(base + kHeaderBytes);
+    o.ms = reinterpret_cast<float2*>(base + kHeaderBytes + ws_keys_bytes(M, k));
+    o.M = M;
+    o.k = k;
+    o.Vt = Vt;
+    return o;
+}
+
+// M at or below which the CUDA-core GEMV is used when both paths can run the shape.
+constexpr int kGemvMaxM = 4;
+
+static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
+    if (path == VT_PATH_GEMV) return launch_head_gemv(c, st);
+    if (path == VT_PATH_MMA) return launch_head_mma(c, st);
+    if (path != VT_PATH_AUTO) return VT_ERR_SHAPE;
+    if (c.M <= kGemvMaxM && gemv_supports(c.d)) return launch_head_gemv(c, st);
+    vt_status r = launch_head_mma(c, st);
+    if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st);
+    return r;
+}
+
+}  // namespace vt
+
+using namespace vt;
+
+extern "C" {
+
+const char* vt_strerror(vt_status s) {
+    switch (s) {
+        case VT_OK: return "ok";
+        case VT_ERR_NULL: return "a required pointer is NULL";
+        case VT_ERR_SHAPE: return "a size or shape argument is outside the supported range";
+        case VT_ERR_ALIGN: return "a pointer is not aligned as required";
+        case VT_ERR_RANGE: return "a keep id lies outside [0, V_full)";
+        case VT_ERR_DUP: return "keep_ids names an id more than once";
+        case VT_ERR_EMPTY: return "coverage of an empty token stream is undefined";
+        case VT_ERR_WORKSPACE: return "workspace is NULL, misaligned or too small";
+        case VT_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case VT_ERR_CUDA: return "a CUDA call failed";
+        case VT_ERR_UNSUPPORTED: return "the forced path cannot run this shape";
+    }
+    return "unknown status";
+}
+
+int vt_last_cuda_error(void) { return g_last_cuda_error; }
+int vt_last_launch_count(void) { return g_launches; }
+
+vt_status vt_compact_head(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim, void* W_trim,
+                          void* stream) {
+    g_launches = 0;
+    if (!W_full || !keep_ids || !W_trim) return VT_ERR_NULL;
+    if (d < 8 || d % 8 != 0 || V_full < 1 || V_trim < 1 || V_trim > V_full) return VT_ERR_SHAPE;
+    if (!aligned(W_full, 16) || !aligned(W_trim, 16) || !aligned(keep_ids, 4)) return VT_ERR_ALIGN;
+    return launch_compact(W_full, V_full, d, keep_ids, V_trim, W_trim, (cudaStream_t)stream);
+}
+
+size_t vt_coverage_workspace_bytes(int V_full) {
+    if (V_full < 1) return 0;
+    size_t b = sizeof(CoverageCounters) + coverage_bitmap_words(V_full) * 4;
+    return (b + 255) & ~(size_t)255;
+}
+
+static vt_status read_counters(void* workspace, cudaStream_t st, CoverageCounters* host) {
+    cudaError_t e = cudaMemcpyAsync(host, workspace, sizeof(CoverageCounters), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+vt_status vt_validate_keep_ids(const int32_t* keep_ids, int V_trim, int V_full, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    g_launches = 0;
+    if (!keep_ids) return VT_ERR_NULL;
+    if (V_full < 1 || V_trim < 1) return VT_ERR_SHAPE;
+    if (!aligned(keep_ids, 4)) return VT_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < vt_coverage_workspace_bytes(V_full))
+        return VT_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    vt_status r = launch_keep_bitmap(keep_ids, V_trim, V_full, workspace, st);
+    if (r != VT_OK) return r;
+    CoverageCounters c;
+    r = read_counters(workspace, st, &c);
+    if (r != VT_OK) return r;
+    if (c.out_of_range) return VT_ERR_RANGE;
+    if (c.duplicates) return VT_ERR_DUP;
+    if (V_trim > V_full) return VT_ERR_SHAPE;   // unreachable for a valid set; kept for completeness
+    return VT_OK;
+}
+
+size_t vt_workspace_bytes(int M, int k) {
+    if (M < 1 || k < 1 || k > VT_MAX_K) return 0;
+    return ws_total_bytes(M, k);
+}
+
+vt_status vt_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < kHeaderBytes) return VT_ERR_WORKSPACE;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream);
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d2t, int M, int d, int V_trim, int k,
+                             int32_t* target_ids, float* logprobs, int32_t* draft_ids, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream, int path) {
+    g_launches = 0;
+    vt_status r = check_head_args(h, W_trim, d2t, M, d, V_trim, k, target_ids, logprobs, workspace, workspace_bytes);
+    if (r != VT_OK) return r;
+    HeadCall c{h, W_trim, d, M, V_trim,
+               make_out(d2t, M, V_trim, k, target_ids, logprobs, draft_ids, lse, nullptr, workspace)};
+    return run_head(c, (cudaStream_t)stream, path);
+}
+
+vt_status vt_draft_head(const void* h, const void* W_trim, const int32_t* d2t, int M, int d, int V_trim, int k,
+                        int32_t* target_ids, float* logprobs, int32_t* draft_ids, float* lse, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    return vt_draft_head_path(h, W_trim, d2t, M, d, V_trim, k, target_ids, logprobs, draft_ids, lse, workspace,
+                              workspace_bytes, stream, VT_PATH_AUTO);
+}
+
+static inline size_t up256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+size_t vt_host_workspace_bytes(int M, int d, int k) {
+    if (M < 1 || k < 1 || k > VT_MAX_K || d < 8) return 0;
+    return ws_total_bytes(M, k) + up256((size_t)M * d * 2) + 2 * up256((size_t)M * k * 4);
+}
+
+vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32_t* d2t, int M, int d, int V_trim,
+                             int k, int32_t* target_ids_host, float* logprobs_host, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    g_launches = 0;
+    if (!h_host || !target_ids_host || !logprobs_host) return VT_ERR_NULL;
+    if (d < 8 || d % 8 != 0 || M < 1 || k < 1 || k > VT_MAX_K) return VT_ERR_SHAPE;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < vt_host_workspace_bytes(M, d, k))
+        return VT_ERR_WORKSPACE;
+    unsigned char* base = reinterpret_cast<unsigned char*>(workspace);
+    const size_t head_ws = ws_total_bytes(M, k);
+    void* h_dev = base + head_ws;
+    int32_t* tid_dev = reinterpret_cast<int32_t*>(base + head_ws + up256((size_t)M * d * 2));
+    float* lp_dev = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(tid_dev) + up256((size_t)M * k * 4));
+    vt_status r = check_head_args(h_dev, W_trim, d2t, M, d, V_trim, k, tid_dev, lp_dev, workspace, head_ws);
+    if (r != VT_OK) return r;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(h_dev, h_host, (size_t)M * d * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    HeadCall c{h_dev, W_trim, d, M, V_trim, make_out(d2t, M, V_trim, k, tid_dev, lp_dev, nullptr, nullptr, nullptr, workspace)};
+    r = run_head(c, st, VT_PATH_AUTO);
+    if (r != VT_OK) return r;
+    e = cudaMemcpyAsync(target_ids_host, tid_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaMemcpyAsync(logprobs_host, lp_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+vt_status vt_last_status(void* workspace, void* stream) {
+    if (!workspace) return VT_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(workspace);
+    unsigned int status = 0;
+    cudaError_t e = cudaMemcpyAsync(&status, &hdr->status, 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (status) {
+        e = cudaMemsetAsync(&hdr->status, 0, 4, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return (status & kStatusTimeout) ? VT_ERR_TIMEOUT : VT_OK;
+}
+
+vt_status vt_coverage(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
+                      uint64_t* covered_out, double* fraction_out, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    g_launches = 0;
+    if (!keep_ids || (!token_ids && N > 0)) return VT_ERR_NULL;
+    if (V_full < 1 || V_trim < 1 || N < 0) return VT_ERR_SHAPE;
+    if (N == 0) return VT_ERR_EMPTY;
+    if (!aligned(token_ids, 4) || !aligned(keep_ids, 4)) return VT_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < vt_coverage_workspace_bytes(V_full))
+        return VT_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    vt_status r = launch_keep_bitmap(keep_ids, V_trim, V_full, workspace, st);
+    if (r != VT_OK) return r;
+    r = launch_coverage_count(token_ids, N, V_full, workspace, st);
+    if (r != VT_OK) return r;
+    CoverageCounters c;
+    r = read_counters(workspace, st, &c);
+    if (r != VT_OK) return r;
+    if (covered_out) *covered_out = c.covered;
+    if (fraction_out) *fraction_out = (double)c.covered / (double)N;
+    return VT_OK;
+}
+
+vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V_trim, float* logits, void* workspace,
+                          size_t workspace_bytes, void* stream, int path) {
+    g_launches = 0;
+    if (!logits) return VT_ERR_NULL;
+    if (!aligned(logits, 4)) return VT_ERR_ALIGN;
+    // the epilogue still runs its top-1 bookkeeping; its outputs land in the tail of the workspace
+    if (M < 1) return VT_ERR_SHAPE;
+    const size_t head_ws = ws_total_bytes(M, 1);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < ws_total_bytes(M, 2)) return VT_ERR_WORKSPACE;
+    unsigned char* base = reinterpret_cast<unsigned char*>(workspace);
+    int32_t* tid = reinterpret_cast<int32_t*>(base + head_ws);
+    float* lp = reinterpret_cast<float*>(base + head_ws + up256((size_t)M * 4));
+    // no d2t here: the merge then reports draft indices; `tid` only stands in for the NULL check
+    vt_status r = check_head_args(h, W_trim, tid, M, d, V_trim, 1, tid, lp, workspace, head_ws);
+    if (r != VT_OK) return r;
+    HeadOut o = make_out(nullptr, M, V_trim, 1, tid, lp, nullptr, nullptr, logits, workspace);
+    HeadCall c{h, W_trim, d, M, V_trim, o};
+    return run_head(c, (cudaStream_t)stream, path);
+}
+
+vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim, int32_t* target_ids,
+                   void* stream) {
+    g_launches = 0;
+    if (!draft_ids || !d2t || !target_ids) return VT_ERR_NULL;
+    if (n < 0 || V_trim < 1) return VT_ERR_SHAPE;
+    if (!aligned(draft_ids, 4) || !aligned(d2t, 4) || !aligned(target_ids, 4)) return VT_ERR_ALIGN;
+    return launch_remap(draft_ids, d2t, n, V_trim, target_ids, (cudaStream_t)stream);
+}
+
+}  // extern "C"

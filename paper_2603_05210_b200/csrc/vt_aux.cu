@@ -1,0 +1,189 @@
+// The memory-bound helpers around the head: row-gather compaction (the draft vocabulary keeps
+// only the rows of V_d), the draft-to-target remap, and the Eq. 2 coverage count.
+#include "vt_launch.h"
+
+namespace vt {
+
+// ------------------------------------------------------------------------------------------
+// W_trim[i, :] = W_full[keep_ids[i], :] in 16-byte chunks; four independent chunks per thread
+// per trip keep enough loads in flight to cover HBM latency.
+// ------------------------------------------------------------------------------------------
+constexpr int kCompactUnroll = 4;
+
+__global__ void __launch_bounds__(256) compact_kernel(const uint4* __restrict__ W_full, int V_full,
+                                                      int chunks_per_row, const int32_t* __restrict__ keep_ids,
+                                                      long long total_chunks, uint4* __restrict__ W_trim) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long e0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; e0 < total_chunks;
+         e0 += stride * kCompactUnroll) {
+        uint4 v[kCompactUnroll];
+        bool ok[kCompactUnroll];
+#pragma unroll
+        for (int u = 0; u < kCompactUnroll; ++u) {
+            const long long e = e0 + u * stride;
+            ok[u] = false;
+            if (e < total_chunks) {
+                const int row = (int)(e / chunks_per_row);
+                const int col = (int)(e - (long long)row * chunks_per_row);
+                const int src = __ldg(&keep_ids[row]);
+                if (src >= 0 && src < V_full) {
+                    v[u] = __ldcs(&W_full[(size_t)src * chunks_per_row + col]);
+                    ok[u] = true;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kCompactUnroll; ++u)
+            if (ok[u]) __stcs(&W_trim[e0 + u * stride], v[u]);
+    }
+}
+
+vt_status launch_compact(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim,
+                         void* W_trim, cudaStream_t st) {
+    int sms = 0;
+    vt_status rs = device_sm_count(&sms);
+    if (rs != VT_OK) return rs;
+    const int cpr = d / 8;
+    const long long total = (long long)V_trim * cpr;
+    const long long want = (total + 256LL * kCompactUnroll - 1) / (256LL * kCompactUnroll);
+    const int grid = (int)std::max(1LL, std::min(want, (long long)sms * 8));
+    compact_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const uint4*>(W_full), V_full, cpr, keep_ids, total,
+                                         reinterpret_cast<uint4*>(W_trim));
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
+// target_ids[t] = d2t[draft_ids[t]]
+// ------------------------------------------------------------------------------------------
+__global__ void remap_kernel(const int32_t* __restrict__ draft_ids, const int32_t* __restrict__ d2t, long long n,
+                             int V_trim, int32_t* __restrict__ target_ids) {
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += (long long)gridDim.x * blockDim.x) {
+        const int i = draft_ids[t];
+        target_ids[t] = (i >= 0 && i < V_trim) ? __ldg(&d2t[i]) : -1;
+    }
+}
+
+vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim, int32_t* target_ids,
+                       cudaStream_t st) {
+    if (n == 0) return VT_OK;
+    const int grid = (int)std::min<long long>((n + 255) / 256, 1184);
+    remap_kernel<<<grid, 256, 0, st>>>(draft_ids, d2t, n, V_trim, target_ids);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
+// Membership bitmap of the kept set (bit v of the bitmap = "v is in V_d"); the same pass counts
+// out-of-range ids and ids seen twice.
+// ------------------------------------------------------------------------------------------
+__global__ void keep_bitmap_kernel(const int32_t* __restrict__ keep_ids, int V_trim, int V_full,
+                                   CoverageCounters* counters, unsigned int* bitmap) {
+    unsigned int oor = 0, dup = 0;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < V_trim; i += gridDim.x * blockDim.x) {
+        const int v = keep_ids[i];
+        if (v < 0 || v >= V_full) {
+            ++oor;
+        } else {
+            const unsigned int bit = 1u << (v & 31);
+            if (atomicOr(&bitmap[v >> 5], bit) & bit) ++dup;
+        }
+    }
+    if (oor) atomicAdd(&counters->out_of_range, oor);
+    if (dup) atomicAdd(&counters->duplicates, dup);
+}
+
+vt_status launch_keep_bitmap(const int32_t* keep_ids, int V_trim, int V_full, void* workspace, cudaStream_t st) {
+    const size_t bytes = sizeof(CoverageCounters) + coverage_bitmap_words(V_full) * 4;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, bytes, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    auto* counters = reinterpret_cast<CoverageCounters*>(workspace);
+    auto* bitmap = reinterpret_cast<unsigned int*>(counters + 1);
+    const int grid = std::max(1, std::min((V_trim + 255) / 256, 592));
+    keep_bitmap_kernel<<<grid, 256, 0, st>>>(keep_ids, V_trim, V_full, counters, bitmap);
+    count_launch();
+    e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
+// covered = #{t : token_ids[t] in V_d}: each CTA copies the bitmap to shared memory when it
+// fits, streams its share of the ids with 16-byte loads and adds one 64-bit count per CTA.
+// ------------------------------------------------------------------------------------------
+constexpr int kCoverageThreads = 512;
+constexpr size_t kCoverageSmemBitmapMax = 160 * 1024;
+
+__device__ __forceinline__ unsigned int member(const unsigned int* bm, int v, int V_full) {
+    return ((unsigned int)v < (unsigned int)V_full) ? ((bm[v >> 5] >> (v & 31)) & 1u) : 0u;
+}
+
+__global__ void __launch_bounds__(kCoverageThreads) coverage_count_kernel(
+    const int32_t* __restrict__ token_ids, long long N, int V_full, const unsigned int* __restrict__ bitmap_g,
+    int bitmap_words, int bitmap_in_smem, CoverageCounters* counters) {
+    extern __shared__ unsigned int bm_s[];
+    __shared__ unsigned int warp_counts[kCoverageThreads / 32];
+    const unsigned int* bm = bitmap_g;
+    if (bitmap_in_smem) {
+        for (int w = threadIdx.x; w < bitmap_words; w += blockDim.x) bm_s[w] = bitmap_g[w];
+        __syncthreads();
+        bm = bm_s;
+    }
+    // elements before the first 16-byte boundary and after the last full vector are taken singly
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(token_ids);
+    long long head = (long long)(((16 - (addr & 15)) & 15) / 4);
+    if (head > N) head = N;
+    const long long nvec = (N - head) / 4;
+    const long long tail_begin = head + nvec * 4;
+    const int4* vec = reinterpret_cast<const int4*>(token_ids + head);
+
+    unsigned int c = 0;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long gstride = (long long)gridDim.x * blockDim.x;
+    for (long long i = gtid; i < nvec; i += gstride) {
+        const int4 t = __ldcs(&vec[i]);
+        c += member(bm, t.x, V_full) + member(bm, t.y, V_full) + member(bm, t.z, V_full) + member(bm, t.w, V_full);
+    }
+    for (long long i = gtid; i < head; i += gstride) c += member(bm, token_ids[i], V_full);
+    for (long long i = tail_begin + gtid; i < N; i += gstride) c += member(bm, token_ids[i], V_full);
+
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0) warp_counts[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long total = 0;
+        for (int w = 0; w < kCoverageThreads / 32; ++w) total += warp_counts[w];
+        if (total) atomicAdd(&counters->covered, total);
+    }
+}
+
+vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full, void* workspace, cudaStream_t st) {
+    int sms = 0;
+    vt_status rs = device_sm_count(&sms);
+    if (rs != VT_OK) return rs;
+    auto* counters = reinterpret_cast<CoverageCounters*>(workspace);
+    auto* bitmap = reinterpret_cast<unsigned int*>(counters + 1);
+    const size_t words = coverage_bitmap_words(V_full);
+    const int in_smem = words * 4 <= kCoverageSmemBitmapMax;
+    const size_t smem = in_smem ? words * 4 : 0;
+    static int configured_device = -1;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    if (configured_device != dev) {
+        cudaError_t e = cudaFuncSetAttribute(coverage_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kCoverageSmemBitmapMax);
+        if (e != cudaSuccess) return cuda_fail(e);
+        configured_device = dev;
+    }
+    const long long per_cta = (long long)kCoverageThreads * 4 * 8;   // ids one CTA takes in 8 trips
+    const int grid = (int)std::max(1LL, std::min((N + per_cta - 1) / per_cta, (long long)sms * 2));
+    coverage_count_kernel<<<grid, kCoverageThreads, smem, st>>>(token_ids, N, V_full, bitmap, (int)words, in_smem,
+                                                               counters);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+}  // namespace vt

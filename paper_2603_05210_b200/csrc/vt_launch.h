@@ -1,0 +1,48 @@
+// Host-side glue shared by the kernel launchers and the C entry points.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+
+#include "vt_common.cuh"
+
+namespace vt {
+
+constexpr int kMaxDynSmem = 227 * 1024;   // opt-in dynamic shared memory per CTA on sm_100
+
+// One draft-head call after validation (all pointers device).
+struct HeadCall {
+    const void* h;
+    const void* W;
+    int d, M, Vt;
+    HeadOut out;
+};
+
+vt_status cuda_fail(cudaError_t e);        // records e for vt_last_cuda_error, returns VT_ERR_CUDA
+vt_status driver_fail(int cu_result);
+void count_launch();
+vt_status device_sm_count(int* sms);
+
+bool gemv_supports(int d);
+vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st);
+vt_status launch_head_mma(const HeadCall& c, cudaStream_t st);
+
+vt_status launch_compact(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim,
+                         void* W_trim, cudaStream_t st);
+vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
+                       int32_t* target_ids, cudaStream_t st);
+
+// Coverage workspace: one 256-byte line of counters, then the membership bitmap.
+struct CoverageCounters {
+    unsigned long long covered;
+    unsigned int out_of_range;
+    unsigned int duplicates;
+    unsigned int pad[60];
+};
+static_assert(sizeof(CoverageCounters) == 256, "one line");
+inline size_t coverage_bitmap_words(int V_full) { return ((size_t)V_full + 31) / 32; }
+vt_status launch_keep_bitmap(const int32_t* keep_ids, int V_trim, int V_full, void* workspace, cudaStream_t st);
+vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full, void* workspace, cudaStream_t st);
+
+}  // namespace vt

@@ -1,0 +1,211 @@
+"""CUDA kernels vs the CPU oracle, element by element, on shapes the oracle finishes in seconds.
+
+Shapes span several tiles and ragged tails: vocabulary sizes that are not multiples of any tile
+(1, 7, 127, 129, 4380, 6521 - the paper's in-domain draft vocabularies, Section 3.2), hidden sizes
+from one 16-byte chunk up to 5120, and draft-row counts across the per-pass limits of both paths.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_05210_b200 import inputs
+from tests import parity
+from tests.gpu_util import Guarded, dev_bf16, dev_i32, run_head
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def vt():
+    import paper_2603_05210_b200 as vt
+    vt.lib()
+    assert torch.cuda.is_available()
+    return vt
+
+
+def rand_case(M, d, Vt, seed, w_std=0.02, h_std=1.0):
+    rng = np.random.default_rng(seed)
+    W = inputs.f32_to_bf16_bits((w_std * rng.standard_normal((Vt, d))).astype(np.float32)).reshape(Vt, d)
+    h = inputs.f32_to_bf16_bits((h_std * rng.standard_normal((M, d))).astype(np.float32)).reshape(M, d)
+    d2t = rng.permutation(max(Vt * 3, 10))[:Vt].astype(np.int32)
+    return h, W, d2t
+
+
+PATHS = [pytest.param(1, id="gemv"), pytest.param(2, id="mma")]
+
+
+# ------------------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("V,d,Vt", [(50, 8, 1), (300, 64, 77), (1000, 2048, 129), (5000, 5120, 4380), (257, 24, 257)])
+def test_compact_head_bit_exact(vt, oracle, V, d, Vt):
+    rng = np.random.default_rng(V + d)
+    W = rng.integers(0, 2 ** 16, size=(V, d), dtype=np.uint16)
+    keep = rng.permutation(V)[:Vt].astype(np.int32)
+    out = Guarded((Vt, d), torch.bfloat16)
+    vt.vt_compact_head(dev_bf16(W), dev_i32(keep), out=out.t)
+    torch.cuda.synchronize()
+    got = out.t.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, oracle.compact(W, keep))
+    assert out.intact()
+
+
+# ------------------------------------------------------------------------------ coverage (Eq. 2)
+@pytest.mark.parametrize("V,N,Vt,offset", [(50, 1, 5, 0), (1000, 4099, 100, 1), (128256, 300_001, 13264, 3),
+                                           (128256, 40_850, 4380, 2), (7_000_000, 50_000, 100_000, 0)])
+def test_coverage_bit_exact(vt, oracle, V, N, Vt, offset):
+    rng = np.random.default_rng(N)
+    tok = rng.integers(-3, V + 3, size=N + offset).astype(np.int32)     # a few ids fall outside [0, V)
+    keep = rng.permutation(V)[:Vt].astype(np.int32)
+    tok_dev = dev_i32(tok)[offset:]                                       # start off a 16-byte boundary
+    covered, frac = vt.vt_coverage(tok_dev, dev_i32(keep), V)
+    assert (covered, frac) == oracle.coverage(tok[offset:], keep, V)
+
+
+def test_coverage_zipf_stream_and_validate(vt, oracle):
+    V = inputs.V_LLAMA3
+    tok = inputs.zipf_token_stream(V, 1.1, 574_168, seed=2)               # combined size of Table 4's streams
+    order, _ = inputs.frequency_ranking(tok, V)
+    tok_dev = dev_i32(tok)
+    for Vt in (4380, 6521, 13264, V):
+        assert vt.vt_coverage(tok_dev, dev_i32(order[:Vt]), V) == oracle.coverage(tok, order[:Vt], V)
+    assert vt.vt_validate_keep_ids(dev_i32(order[:13264]), V) == vt.VT_OK
+    dup = order[:100].copy()
+    dup[57] = dup[3]
+    assert vt.vt_validate_keep_ids(dev_i32(dup), V) == vt.VT_ERR_DUP
+    oor = order[:100].copy()
+    oor[99] = V
+    assert vt.vt_validate_keep_ids(dev_i32(oor), V) == vt.VT_ERR_RANGE
+    with pytest.raises(vt.VtError) as e:
+        vt.vt_coverage(tok_dev[:0], dev_i32(order[:10]), V)
+    assert e.value.status == vt.VT_ERR_EMPTY
+
+
+# ------------------------------------------------------------------------------ remap
+def test_remap_bit_exact(vt, oracle):
+    rng = np.random.default_rng(3)
+    d2t = rng.permutation(128256)[:4380].astype(np.int32)
+    idx = rng.integers(0, 4380, size=(17, 10)).astype(np.int32)
+    got = vt.vt_remap(dev_i32(idx), dev_i32(d2t)).cpu().numpy()
+    assert np.array_equal(got, oracle.remap(idx, d2t))
+    bad = idx.copy()
+    bad[0, 0], bad[1, 1] = -1, 4380
+    got = vt.vt_remap(dev_i32(bad), dev_i32(d2t)).cpu().numpy()
+    assert got[0, 0] == -1 and got[1, 1] == -1 and np.array_equal(got[2:], oracle.remap(idx, d2t)[2:])
+
+
+# ------------------------------------------------------------------------------ logits
+LOGIT_SHAPES = [(1, 8, 1), (1, 64, 7), (3, 64, 127), (8, 2048, 129), (2, 3072, 1000), (4, 4096, 4380),
+                (9, 2048, 300), (17, 64, 1025), (3, 5120, 700), (5, 200, 2000), (64, 512, 333), (1, 8192, 150)]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,d,Vt", LOGIT_SHAPES)
+def test_logits_vs_oracle(vt, oracle, path, M, d, Vt):
+    h, W, _ = rand_case(M, d, Vt, seed=M * 1000 + Vt)
+    got = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=path).cpu().numpy()
+    parity.check_logits(got, oracle.logits(h, W))
+
+
+# ------------------------------------------------------------------------------ full head
+HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8), (8, 2048, 129, 10),
+               (8, 4096, 6521, 8), (2, 3072, 1000, 64), (9, 2048, 300, 10), (17, 128, 1025, 3),
+               (4, 5120, 700, 8), (64, 512, 333, 10), (5, 200, 2000, 33), (1, 4096, 13264, 1)]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,d,Vt,k", HEAD_SHAPES)
+def test_draft_head_vs_oracle(vt, oracle, path, M, d, Vt, k):
+    h, W, d2t = rand_case(M, d, Vt, seed=M * 77 + Vt + k)
+    ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
+    got = run_head(vt, h, dev_bf16(W), d2t, k, path)
+    parity.check_head(got, ora, d2t, k)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_large_logits_keep_softmax_stable(vt, oracle, path):
+    # |x| in the hundreds: exp() of a raw logit would overflow fp32, the running max must absorb it
+    h, W, d2t = rand_case(4, 256, 900, seed=5, w_std=1.0, h_std=8.0)
+    ora = oracle.draft_head(h, W, d2t, 5, want_logits=True)
+    assert np.abs(ora["logits"]).max() > 200
+    got = run_head(vt, h, dev_bf16(W), d2t, 5, path)
+    assert np.all(np.isfinite(got["logprobs"]))
+    # at this magnitude fp32 accumulation error scales with |x|; ids must still match where gaps are wide
+    x = ora["logits"]
+    for m in range(4):
+        assert got["draft_ids"][m, 0] == ora["draft_ids"][m, 0] or \
+            abs(x[m, got["draft_ids"][m, 0]] - x[m, ora["draft_ids"][m, 0]]) < 2e-3 * np.abs(x[m]).max()
+    assert np.max(np.abs(got["lse"] - ora["lse"])) <= 2e-3 * np.abs(ora["lse"]).max()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_exact_ties_resolve_to_lowest_draft_index(vt, oracle, path):
+    # duplicated weight rows give bit-equal logits on both sides
+    rng = np.random.default_rng(8)
+    M, d, Vt, k = 3, 256, 600, 10
+    base = inputs.f32_to_bf16_bits((0.05 * rng.standard_normal((60, d))).astype(np.float32)).reshape(60, d)
+    W = base[rng.integers(0, 60, size=Vt)]
+    h = inputs.f32_to_bf16_bits(rng.standard_normal((M, d)).astype(np.float32)).reshape(M, d)
+    d2t = np.arange(Vt, dtype=np.int32) + 1000
+    ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
+    got = run_head(vt, h, dev_bf16(W), d2t, k, path)
+    assert np.array_equal(got["draft_ids"], ora["draft_ids"])
+    assert np.array_equal(got["target_ids"], ora["target_ids"])
+    parity.check_exact_tie_order(got["draft_ids"], ora["logits"])
+    # zero hidden state: every logit is 0, the winners are indices 0..k-1, log-prob = -log(Vt)
+    h0 = np.zeros((2, d), dtype=np.uint16)
+    got0 = run_head(vt, h0, dev_bf16(W), d2t, k, path)
+    assert np.array_equal(got0["draft_ids"], np.tile(np.arange(k, dtype=np.int32), (2, 1)))
+    assert np.allclose(got0["logprobs"], -np.log(Vt), atol=1e-5)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_same_input_twice_is_bit_identical_and_workspace_is_reusable(vt, oracle, path):
+    h, W, d2t = rand_case(8, 1024, 5000, seed=9)
+    Wd = dev_bf16(W)
+    ws = vt.new_workspace(vt.vt_workspace_bytes(8, 8))
+    a = run_head(vt, h, Wd, d2t, 8, path, workspace=ws)
+    b = run_head(vt, h, Wd, d2t, 8, path, workspace=ws)
+    for key in a:
+        assert np.array_equal(a[key].view(np.int32), b[key].view(np.int32)), key
+    # a different, smaller call on the same workspace afterwards
+    h2, W2, d2t2 = rand_case(2, 64, 50, seed=10)
+    got = run_head(vt, h2, dev_bf16(W2), d2t2, 3, path, workspace=ws)
+    parity.check_head(got, oracle.draft_head(h2, W2, d2t2, 3, want_logits=True), d2t2, 3)
+
+
+def test_both_paths_agree_on_logits(vt):
+    h, W, _ = rand_case(8, 4096, 2000, seed=11)
+    a = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=1).cpu().numpy()
+    b = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=2).cpu().numpy()
+    assert np.max(np.abs(a - b)) <= 2e-3
+
+
+def test_trimmed_head_equals_full_head_restricted(vt, oracle):
+    # the invariant trimming rests on, end to end on the GPU: compact + head over V_d == full head restricted to V_d
+    V, d, M, Vt, k = 3000, 512, 4, 700, 8
+    rng = np.random.default_rng(12)
+    W_full = inputs.f32_to_bf16_bits((0.02 * rng.standard_normal((V, d))).astype(np.float32)).reshape(V, d)
+    h = inputs.f32_to_bf16_bits(rng.standard_normal((M, d)).astype(np.float32)).reshape(M, d)
+    keep = rng.permutation(V)[:Vt].astype(np.int32)
+    W_trim = vt.vt_compact_head(dev_bf16(W_full), dev_i32(keep))
+    got = run_head(vt, h, W_trim, keep, k, 0)
+    full = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W_full)).cpu().numpy()
+    trim = vt.vt_debug_logits(dev_bf16(h), W_trim).cpu().numpy()
+    assert np.array_equal(trim, full[:, keep])                       # same products, same order: bit-equal
+    ora = oracle.draft_head(h, oracle.compact(W_full, keep), keep, k, want_logits=True)
+    parity.check_head(got, ora, keep, k)
+    ident = np.arange(V, dtype=np.int32)
+    got_full = run_head(vt, h, dev_bf16(W_full), ident, 1, 0)
+    assert np.array_equal(got_full["target_ids"], got_full["draft_ids"])
+    assert np.array_equal(got_full["target_ids"][:, 0], np.argmax(oracle.logits(h, W_full), axis=1))
+
+
+def test_host_buffer_entry_point(vt, oracle):
+    M, d, Vt, k = 8, 1024, 3000, 8
+    h, W, d2t = rand_case(M, d, Vt, seed=13)
+    ws = vt.new_workspace(vt.vt_host_workspace_bytes(M, d, k))
+    h_host = torch.from_numpy(h.view(np.int16)).pin_memory()
+    tid = torch.empty((M, k), dtype=torch.int32).pin_memory()
+    lp = torch.empty((M, k), dtype=torch.float32).pin_memory()
+    vt.vt_draft_head_host(h_host, dev_bf16(W), dev_i32(d2t), k, tid, lp, ws)
+    ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
+    parity.check_head({"target_ids": tid.numpy(), "logprobs": lp.numpy()}, ora, d2t, k)
