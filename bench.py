@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the trimmed-vocabulary draft head on B200.
+
+One step = one ``vt_draft_head`` call (contraction, top-k, log-softmax, d2t remap: one launch) on the
+workload ``d=4096, V_trim=32000 of V_full=128256, M=8, k=8``.  The once-per-model steps (head
+compaction, coverage of the token stream) are timed separately and reported under ``once_per_model``.
+Inputs are synthetic and seeded.  Successive calls rotate over enough copies of ``W_trim`` that every
+call streams its weights from HBM rather than from L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-curve]
+
+prints one JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_05210_b200 import inputs  # noqa: E402
+
+METRIC = "draft_head_us_per_call"
+UNIT = "us/call"
+WORKLOAD = dict(d=4096, V_full=inputs.V_LLAMA3, V_trim=32000, M=8, k=8, seed=3000)
+WORKLOAD_NAME = "d=4096, V_trim=32000 of V_full=128256, M=8, top-k=8, log-softmax over V_trim, d2t remap"
+CURVE_VT = (4096, 8192, 16384, 32000, 128256)
+CURVE_M = (1, 2, 4, 8, 16, 32, 64)
+FALLBACK_HBM_GBS = 6650.0
+
+
+def head_bytes(d, Vt, M, k):
+    """Algorithmic bytes of one call: weights once, hidden states, d2t gathers and both outputs."""
+    return 2 * d * Vt + 2 * M * d + M * k * 12
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def to_dev(a, torch, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.view(dtype) if dtype is not None else t
+
+
+def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0):
+    """CUDA-event time of `steps` back-to-back calls rotating over W_copies; returns ms total."""
+    M = h.shape[0]
+    ws = vt.new_workspace(vt.vt_workspace_bytes(M, k))
+    tid = torch.empty((M, k), dtype=torch.int32, device="cuda")
+    lp = torch.empty((M, k), dtype=torch.float32, device="cuda")
+    n = len(W_copies)
+    for i in range(warmup):
+        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(steps):
+        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+    e1.record()
+    torch.cuda.synchronize()
+    assert vt.vt_last_status(ws) == vt.VT_OK, "a device-side wait ran out during the timed region"
+    return e0.elapsed_time(e1), vt.vt_last_launch_count()
+
+
+def n_copies_for_cold(bytes_per_copy, l2_bytes, free_bytes):
+    want = max(2, -(-4 * l2_bytes // bytes_per_copy))
+    return int(max(1, min(want, (free_bytes // 2) // bytes_per_copy)))
+
+
+def run_ours(args):
+    import torch
+
+    import paper_2603_05210_b200 as vt
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the draft head")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    vt.lib()
+    props = torch.cuda.get_device_properties(local)
+    l2 = int(props.L2_cache_size)
+    peak_gbs, peak_kind = measured_peaks()
+
+    w = WORKLOAD
+    d, V, Vt, M, k = w["d"], w["V_full"], w["V_trim"], w["M"], w["k"]
+    tokens = inputs.zipf_token_stream(V, 1.1, 1_000_000, w["seed"])
+    ranking = inputs.frequency_ranking(tokens, V)
+    case = inputs.make_case("bench", d, Vt, M, k, w["seed"], row_scale=(0.5, 2.0), ranking=ranking)
+    W_full = to_dev(case.W_full.view(np.int16), torch, torch.bfloat16)
+    keep = to_dev(case.keep_ids, torch)
+    d2t = to_dev(case.d2t, torch)
+    h = to_dev(case.h.view(np.int16), torch, torch.bfloat16)
+    tok_dev = to_dev(tokens, torch)
+
+    # once-per-model steps: compaction (a1) and coverage (a6)
+    W_trim = vt.vt_compact_head(W_full, keep)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(10):
+        vt.vt_compact_head(W_full, keep, out=W_trim)
+    e1.record()
+    torch.cuda.synchronize()
+    compact_us = e0.elapsed_time(e1) * 100.0
+    cov_ws = torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda")
+    vt.vt_coverage(tok_dev, keep, V, cov_ws)
+    t0 = time.perf_counter()
+    for _ in range(10):
+        covered, frac = vt.vt_coverage(tok_dev, keep, V, cov_ws)
+    coverage_us = (time.perf_counter() - t0) * 1e5
+
+    free, _ = torch.cuda.mem_get_info()
+    nc = n_copies_for_cold(W_trim.numel() * 2, l2, free)
+    copies = [W_trim] + [W_trim.clone() for _ in range(nc - 1)]
+
+    # ---- timed region: K calls, device-timed, max over ranks
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ms, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup)
+    clocks = sampler.stop()
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        dist.barrier()
+    us_per_call_rank = ms * 1000.0 / args.steps
+    value = us_per_call_rank / world                  # whole job: N replicas finish N calls in that time
+    bytes_call = head_bytes(d, Vt, M, k)
+    achieved = bytes_call / (us_per_call_rank * 1e-6) / 1e9
+
+    # ---- end to end: host h -> device, head, outputs -> host, every step
+    e2e_steps = max(1, min(args.steps, 2000))
+    hws = vt.new_workspace(vt.vt_host_workspace_bytes(M, d, k))
+    h_host = torch.from_numpy(case.h.view(np.int16).copy()).pin_memory()
+    tid_h = torch.empty((M, k), dtype=torch.int32).pin_memory()
+    lp_h = torch.empty((M, k), dtype=torch.float32).pin_memory()
+    for i in range(min(args.warmup, 50)):
+        vt.vt_draft_head_host(h_host, copies[i % nc], d2t, k, tid_h, lp_h, hws)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        vt.vt_draft_head_host(h_host, copies[i % nc], d2t, k, tid_h, lp_h, hws)
+    e2e_us = (time.perf_counter() - t0) * 1e6 / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_us], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item())
+
+    line = {
+        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 6), "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAME, "cold": f"calls rotate over {nc} copies of W_trim "
+                   f"({nc * W_trim.numel() * 2 / 1e6:.0f} MB >= 4x L2 of {l2 / 1e6:.0f} MB): inputs larger than L2",
+                   "step": "one vt_draft_head call (contraction + top-k + log-softmax + remap, one launch)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "calls_per_s": round(1e6 / value, 1)},
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
+                     "frac": round(achieved / peak_gbs, 4), "of": peak_kind, "traffic": None,
+                     "algorithmic_bytes_per_launch": bytes_call, "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
+                     "kernel": "head kernel of the chosen path; duration = timed region / launches"},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_us / world, 3), "unit": UNIT, "h2d_bytes_per_step": M * d * 2,
+                "d2h_bytes_per_step": M * k * 8, "steps": e2e_steps},
+        "gpu_launches": args.steps * launches_per_call,
+        "once_per_model": {"compact_us": round(compact_us, 2),
+                           "compact_GBs": round(2 * W_trim.numel() * 2 / compact_us / 1e3, 1),
+                           "coverage_us_incl_sync": round(coverage_us, 2), "coverage_tokens": int(tokens.size),
+                           "coverage": frac},
+    }
+
+    if rank == 0 and world == 1:
+        if not args.no_curve:
+            line["curve"] = latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs)
+        line["cpu_baseline"] = cpu_baseline(case)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs):
+    """us/call and roofline fraction over V_trim x M at d=4096 (the measured latency-vs-vocabulary curve)."""
+    d, k = case.d, 8
+    order = ranking[0]
+    out = []
+    for Vt in CURVE_VT:
+        keep = to_dev(np.ascontiguousarray(order[:Vt]), torch)
+        W_trim = vt.vt_compact_head(W_full, keep)
+        free, _ = torch.cuda.mem_get_info()
+        nc = n_copies_for_cold(W_trim.numel() * 2, l2, free)
+        copies = [W_trim] + [W_trim.clone() for _ in range(nc - 1)]
+        for M in CURVE_M:
+            h = to_dev(inputs.hidden_states_bf16(M, d, 77 + M).view(np.int16), torch, torch.bfloat16)
+            kk = min(k, Vt)
+            steps = 400 if Vt <= 32000 else 100
+            ms, _ = time_head(vt, torch, h, copies, keep, kk, steps, 20)
+            us = ms * 1000.0 / steps
+            gbs = head_bytes(d, Vt, M, kk) / (us * 1e-6) / 1e9
+            out.append({"V_trim": Vt, "M": M, "us_per_call": round(us, 2), "GBs": round(gbs, 1),
+                        "frac": round(gbs / peak_gbs, 4)})
+        del copies, W_trim
+        torch.cuda.empty_cache()
+    return out
+
+
+def cpu_baseline(case):
+    """The oracle as it stands, timed on this host on the bench workload (best of 3 full calls)."""
+    import oracle
+    W_trim = oracle.compact(case.W_full, case.keep_ids)
+    best = float("inf")
+    for _ in range(3):
+        t0 = time.perf_counter()
+        oracle.draft_head(case.h, W_trim, case.d2t, case.k)
+        best = min(best, time.perf_counter() - t0)
+    return {"value": round(best * 1e6, 1), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "the whole bench workload, one full call, best of 3"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the same workload and metric (a deliberately plain program)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = WORKLOAD
+    d, V, Vt, M, k = w["d"], w["V_full"], w["V_trim"], w["M"], w["k"]
+    tokens = inputs.zipf_token_stream(V, 1.1, 1_000_000, w["seed"])
+    ranking = inputs.frequency_ranking(tokens, V)
+    # weights only for the sampled rows: the oracle's cost per row does not depend on their values' origin
+    rng_rows = 2048
+    case = inputs.make_case("ref", d, rng_rows, M, k, w["seed"], V_full=V, ranking=ranking,
+                            W_full=inputs.normal_bf16((rng_rows, d), 0.02, w["seed"]),
+                            row_scale=(0.5, 2.0))
+    W = case.W_full
+    d2t = np.ascontiguousarray(ranking[0][:rng_rows])
+    t0 = time.perf_counter()
+    oracle.draft_head(case.h, W, d2t, k)
+    probe = time.perf_counter() - t0
+    per_row = probe / rng_rows
+    total_steps = args.steps + args.warmup
+    rows = int(max(256, min(Vt, 120.0 / max(total_steps, 1) / per_row)))
+    if rows > rng_rows:
+        W = inputs.normal_bf16((rows, d), 0.02, w["seed"])
+        d2t = np.ascontiguousarray(ranking[0][:rows])
+    else:
+        W, d2t = W[:rows], d2t[:rows]
+    for _ in range(args.warmup):
+        oracle.draft_head(case.h, W, d2t, min(k, rows))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.draft_head(case.h, W, d2t, min(k, rows))
+    dt = (time.perf_counter() - t0) / args.steps
+    us_full = dt * 1e6 * Vt / rows
+    line = {"impl": "reference", "metric": METRIC, "value": round(us_full, 1), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 4),
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAME},
+            "cpu_baseline": {"value": round(us_full, 1), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": f"each step runs the oracle on the first {rows} of {Vt} vocabulary rows "
+                                       f"(all {M} draft rows); value scaled by {Vt}/{rows}"},
+            "e2e": {"value": round(us_full, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-curve", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -168,34 +168,28 @@ __device__ __forceinline__ float warp_sum_f32(float v) {
 
 // ------------------------------------------------------------------------------------------
 // Cross-CTA merge of one draft row by one warp.
-//   P partial lists (descending, k keys each, 0-padded) at keys[(p * M + m) * k + j] and
-//   P pairs (mx_p, s_p) at ms[p * M + m].  `stage` is warp-private shared memory for P * k keys.
+//   P partial lists (descending, k keys each, 0-padded) and
+//   P pairs (mx_p, s_p); both already staged in shared memory: stage[p * k + j], stage_ms[p].
 // Writes the row's k winners in descending key order with their log-probs and target ids.
 // ------------------------------------------------------------------------------------------
 constexpr int kMergeSlots = kMaxParts / 32;
 
-__device__ inline void merge_row(const HeadOut& o, int P, int m, unsigned long long* stage) {
+__device__ inline void merge_row(const HeadOut& o, int P, int m, const unsigned long long* stage,
+                                 const float2* stage_ms) {
     const int lane = threadIdx.x & 31;
-    const int k = o.k, M = o.M;
+    const int k = o.k;
 
     // log-sum-exp over the partials: lse = mx + log sum_p s_p * exp(mx_p - mx)
     float mx = -INFINITY;
-    for (int p = lane; p < P; p += 32) mx = fmaxf(mx, __ldcg(&o.ms[(size_t)p * M + m]).x);
+    for (int p = lane; p < P; p += 32) mx = fmaxf(mx, stage_ms[p].x);
     mx = warp_max_f32(mx);
     float s = 0.0f;
     for (int p = lane; p < P; p += 32) {
-        float2 v = __ldcg(&o.ms[(size_t)p * M + m]);
+        const float2 v = stage_ms[p];
         if (v.y > 0.0f) s += v.y * __expf(v.x - mx);
     }
     s = warp_sum_f32(s);
     const float lse = mx + logf(s);
-
-    // stage all candidate keys (one coalesced pass over L2)
-    for (int p = 0; p < P; ++p) {
-        const unsigned long long* src = o.keys + ((size_t)p * M + m) * k;
-        for (int j = lane; j < k; j += 32) stage[p * k + j] = __ldcg(src + j);
-    }
-    __syncwarp();
 
     // lane owns lists lane, lane+32, ...; every list is sorted, so its best is its head
     int head[kMergeSlots];
@@ -235,7 +229,6 @@ __device__ inline void merge_row(const HeadOut& o, int P, int m, unsigned long l
         }
     }
     if (lane == 0 && o.lse) o.lse[m] = lse;
-    __syncwarp();
 }
 
 // Publishes this CTA's partials (already written to global memory by the calling threads) and
@@ -252,22 +245,52 @@ __device__ inline bool publish_and_check_last(WsHeader* hdr, int* smem_flag) {
     return *smem_flag != 0;
 }
 
-// Last CTA: merges draft rows [m_begin, m_begin + m_count), warps taking rows in turn.
-// `stage_base` is shared memory the CTA no longer uses; floor(stage_bytes / (P*k*8)) warps work
-// at the same time (the host sizes stage_bytes to at least one warp's share).
+// Last CTA: merges draft rows [m_begin, m_begin + m_count).  All threads first copy the partials of
+// a batch of rows from L2 into shared memory (independent loads, a few per thread), then each warp
+// merges one row at a time out of shared memory.  `stage_base` is shared memory the CTA no longer
+// uses; the host sizes it to hold at least one row: P * (k + 1) * 8 bytes.
 __device__ inline void merge_rows(const HeadOut& o, int P, int m_begin, int m_count,
                                   unsigned char* stage_base, size_t stage_bytes) {
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    const size_t per_warp = (size_t)P * o.k * 8;
-    int active = (int)(stage_bytes / per_warp);
-    if (active > nwarps) active = nwarps;
-    if (active < 1) active = 1;
-    if (warp < active) {
-        unsigned long long* stage = reinterpret_cast<unsigned long long*>(stage_base + (size_t)warp * per_warp);
-        for (int m = m_begin + warp; m < m_begin + m_count; m += active) merge_row(o, P, m, stage);
+    const int k = o.k, M = o.M;
+    const size_t per_row = (size_t)P * (k + 1) * 8;
+    int batch = (int)(stage_bytes / per_row);
+    if (batch < 1) batch = 1;
+    if (batch > m_count) batch = m_count;
+    unsigned long long* skeys = reinterpret_cast<unsigned long long*>(stage_base);
+    float2* sms = reinterpret_cast<float2*>(stage_base + (size_t)batch * P * k * 8);
+    const int Pk = P * k;
+    for (int b0 = 0; b0 < m_count; b0 += batch) {
+        const int nb = min(batch, m_count - b0);
+        const int total = nb * Pk;
+        constexpr int U = 4;
+        for (int e0 = threadIdx.x; e0 < total; e0 += blockDim.x * U) {
+            unsigned long long v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int e = e0 + u * blockDim.x;
+                if (e < total) {
+                    const int r = e / Pk, rem = e - r * Pk;
+                    const int p = rem / k, j = rem - p * k;
+                    v[u] = __ldcg(&o.keys[((size_t)p * M + (m_begin + b0 + r)) * k + j]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int e = e0 + u * blockDim.x;
+                if (e < total) skeys[e] = v[u];
+            }
+        }
+        for (int e = threadIdx.x; e < nb * P; e += blockDim.x) {
+            const int r = e / P, p = e - r * P;
+            sms[e] = __ldcg(&o.ms[(size_t)p * M + (m_begin + b0 + r)]);
+        }
+        __syncthreads();
+        for (int r = warp; r < nb; r += nwarps)
+            merge_row(o, P, m_begin + b0 + r, skeys + (size_t)r * Pk, sms + (size_t)r * P);
+        __syncthreads();
     }
-    __syncthreads();
     if (threadIdx.x == 0) o.hdr->ticket = 0u;   // ready for the next call on this stream
 }
 #endif  // __CUDACC__

@@ -293,7 +293,7 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st) {
         const size_t list_bytes = (size_t)c.out.k * MP * 8;
         const size_t bar_bytes = 0;   // sized below, needs n_stages
         (void)bar_bytes;
-        const size_t merge_bytes = (size_t)grid * c.out.k * 8;
+        const size_t merge_bytes = (size_t)grid * (c.out.k + 1) * 8;
         // stages: as many as fit next to the small buffers, at most 8
         int S = 8;
         size_t ring, total;

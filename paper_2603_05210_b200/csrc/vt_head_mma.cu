@@ -1,6 +1,373 @@
-// Draft head, tensor-core path (placeholder until the tcgen05 kernel lands).
+// Draft head, tensor-core path: the head contraction as a tcgen05 GEMM with TMEM accumulators.
+//
+//   D[m, i] = sum_j h[m, j] * W_trim[i, j]       (the d -> k linear head, 2*d*k FLOPs per draft row)
+//
+// Operand roles: A = h (up to 128 draft rows = the 128 TMEM lanes), B = a tile of NT vocabulary rows
+// of W_trim (K-major as stored), D = fp32 accumulator of 128 lanes x NT columns in tensor memory.
+// With draft rows on the lanes, tcgen05.ld hands every epilogue thread one draft row and a run of
+// consecutive vocabulary logits, so the running (max, sum-exp) and the top-k list are thread-private
+// and need no shuffles.  One persistent CTA per SM owns a contiguous range of vocabulary rows:
+//   warp 4   TMA producer: per 64-column k-step one box of h and one box of W into a shared-memory ring
+//   warp 5   MMA issuer: four K=16 tcgen05.mma per k-step, tcgen05.commit frees the ring slot;
+//            two accumulator buffers in TMEM so the epilogue of tile t overlaps the MMAs of tile t+1
+//   warps 0-3 epilogue: warp q reads TMEM lanes 32q..32q+31 (draft rows), never stores a logit
+// The weight stream is the bound (arithmetic intensity = M FLOP/B), so the design spends its
+// shared memory on bytes in flight rather than on operand reuse.
+#include <cuda.h>
+
+#include "vt_common.cuh"
 #include "vt_launch.h"
 
 namespace vt {
-vt_status launch_head_mma(const HeadCall&, cudaStream_t) { return VT_ERR_UNSUPPORTED; }
+
+constexpr int kMmaThreads = 192;
+constexpr int kBoxK = 64;                    // bf16 elements per k-step = one 128-byte swizzle row
+constexpr uint32_t kABytes = 128 * 128;      // A slot: 128 rows x 128 B (only the pass's rows are copied)
+constexpr int kAccStride = 256;              // TMEM columns between the two accumulator buffers
+
+struct MmaParams {
+    HeadOut out;
+    int m_begin, m_count;     // draft rows of this pass
+    int d;
+    int NT;                   // vocabulary rows per tile (multiple of 16, <= 256)
+    int nk;                   // k-steps per tile
+    int n_stages;
+    uint32_t stage_bytes;     // A slot + B slot, multiple of 1024
+    uint32_t a_tx, b_tx;      // bytes each TMA box delivers
+    uint32_t idesc;
+    uint32_t list_off, bar_off, total_smem;   // offsets from the 1024-aligned base
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128-byte swizzled
+// (the layout a TMA box of 64 bf16 columns writes): 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t desc = 0;
+    desc |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    desc |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle): 1
+    desc |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
+    desc |= (uint64_t)1 << 46;                           // descriptor version of sm_100
+    desc |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return desc;
+}
+
+// ------------------------------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(kMmaThreads, 1)
+head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (base - raw);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int Vt = p.out.Vt, k = p.out.k, M = p.out.M, NT = p.NT, S = p.n_stages, nk = p.nk;
+    const int row_begin = (int)((long long)cta * Vt / G);
+    const int row_end = (int)((long long)(cta + 1) * Vt / G);
+    const int nrows = row_end - row_begin;
+    const int ntiles = (nrows + NT - 1) / NT;
+
+    unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [k][128]
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
+    const uint32_t bar_full = base + p.bar_off, bar_empty = bar_full + 8u * S;
+    const uint32_t bar_accf = bar_empty + 8u * S, bar_acce = bar_accf + 16u, bar_drain = bar_acce + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 5);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* last_flag = const_cast<int*>(abort_flag) + 1;
+
+    const int n_epi_warps = (p.m_count + 31) / 32;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_accf + 8u * b, 1);
+            mbar_init(bar_acce + 8u * b, n_epi_warps);
+        }
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    for (int i = tid; i < k * 128; i += blockDim.x) lists[i] = 0ull;
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto fail = [&]() {
+        *abort_flag = 1;
+        atomicOr(&p.out.hdr->status, kStatusTimeout);
+    };
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int it = 0, issued = 0;
+            bool ok = true;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int row0 = row_begin + t * NT;
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % S, n = it / S;
+                    if (n > 0 && !mbar_wait(bar_empty + 8u * s, (uint32_t)(n - 1) & 1u)) { fail(); ok = false; break; }
+                    if (*abort_flag) { ok = false; break; }
+                    const uint32_t a_dst = base + (uint32_t)s * p.stage_bytes;
+                    mbar_arrive_expect_tx(bar_full + 8u * s, p.a_tx + p.b_tx);
+                    tma_load_2d(a_dst, &tmH, ks * kBoxK, p.m_begin, bar_full + 8u * s);
+                    tma_load_2d(a_dst + kABytes, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
+                    issued = it + 1;
+                }
+            }
+            if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
+                for (int i = max(0, issued - S); i < issued; ++i)
+                    (void)mbar_wait(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int buf = t & 1;
+                if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % S;
+                    if (!mbar_wait(bar_full + 8u * s, (uint32_t)(it / S) & 1u)) { fail(); ok = false; break; }
+                    if (*abort_flag) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = base + (uint32_t)s * p.stage_bytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+                    for (int kk = 0; kk < kBoxK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+                        tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, p.idesc, (ks | kk) != 0);
+                    tc_commit(bar_empty + 8u * s);
+                }
+                if (ok) tc_commit(bar_accf + 8u * buf);
+            }
+            if (*abort_flag) {   // every MMA issued so far must retire before TMEM is freed
+                tc_commit(bar_drain);
+                (void)mbar_wait(bar_drain, 0u);
+            }
+        }
+    } else if (warp < n_epi_warps) {
+        // ------------------------------------------------------------------ epilogue: lane = draft row
+        const int m_local = warp * 32 + lane;
+        const bool live = m_local < p.m_count;
+        float mx = -INFINITY, ssum = 0.0f, thr_x = -INFINITY;
+        unsigned long long* my_list = lists + tid;       // list[j * 128 + tid]
+        int filled = 0;
+        for (int t = 0; t < ntiles; ++t) {
+            const int buf = t & 1;
+            if (!mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u)) { fail(); break; }
+            if (*abort_flag) break;
+            tc_fence_after();
+            const int row0 = row_begin + t * NT;
+            const int ncols = min(NT, row_end - row0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kAccStride);
+            for (int c0 = 0; c0 < ncols; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(taddr + (uint32_t)c0, r);
+                tc_wait_ld();
+                if (live) {
+                    const int nv = min(32, ncols - c0);
+                    float cmax = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (c < nv) cmax = fmaxf(cmax, __uint_as_float(r[c]));
+                    if (cmax > mx) {
+                        ssum *= __expf(mx - cmax);
+                        mx = cmax;
+                    }
+                    float add = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (c < nv) add += __expf(__uint_as_float(r[c]) - mx);
+                    ssum += add;
+                    if (cmax > thr_x || filled < k) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const float x = __uint_as_float(r[c]);
+                            if (c < nv && (x > thr_x || filled < k)) {
+                                const unsigned long long kth = list_insert(my_list, 128, k, make_key(x, row0 + c0 + c));
+                                if (filled < k) ++filled;
+                                if (filled == k) thr_x = key_logit(kth);
+                            }
+                        }
+                    }
+                    if (p.out.logits) {
+                        float* dst = p.out.logits + (size_t)(p.m_begin + m_local) * Vt + row0 + c0;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c < nv) dst[c] = __uint_as_float(r[c]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+        }
+        if (live) {
+            const size_t slot = (size_t)cta * M + p.m_begin + m_local;
+            for (int j = 0; j < k; ++j) p.out.keys[slot * k + j] = my_list[j * 128];
+            p.out.ms[slot] = make_float2(mx, ssum);
+        }
+    }
+
+    // ---------------------------------------------------------------------- publish + merge
+    tc_fence_before();
+    const bool last = publish_and_check_last(p.out.hdr, last_flag);
+    tc_fence_after();
+    if (warp == 5)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    if (last) merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.list_off);   // the ring is free now
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static vt_status get_encode(EncodeTiledFn* out) {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (q != cudaDriverEntryPointSuccess || !ptr) return cuda_fail(cudaErrorSymbolNotFound);
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    *out = fn;
+    return VT_OK;
+}
+
+// bf16 matrix [rows, d] row-major, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, int box_rows) {
+    EncodeTiledFn enc;
+    vt_status r = get_encode(&enc);
+    if (r != VT_OK) return r;
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxK, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    CUresult cr = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, elem,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return cr == CUDA_SUCCESS ? VT_OK : driver_fail((int)cr);
+}
+
+// Tile height: a multiple of 16 in [16, 256] that covers ceil(Vt / grid) rows with the least padding,
+// preferring taller tiles (fewer accumulator hand-overs) among equals.
+static int choose_tile_rows(int rows_per_cta) {
+    int best = 16, best_pad = 1 << 30;
+    for (int nt = 16; nt <= 256; nt += 16) {
+        const int tiles = (rows_per_cta + nt - 1) / nt;
+        const int pad = tiles * nt - rows_per_cta;
+        if (pad < best_pad || (pad == best_pad && nt > best)) {
+            best = nt;
+            best_pad = pad;
+        }
+    }
+    return best;
+}
+
+vt_status launch_head_mma(const HeadCall& c, cudaStream_t st) {
+    int sms = 0;
+    vt_status r = device_sm_count(&sms);
+    if (r != VT_OK) return r;
+    const int grid = std::max(1, std::min(std::min(sms, kMaxParts), (c.Vt + 15) / 16));
+    const int rows_per_cta = (c.Vt + grid - 1) / grid;
+    const int NT = choose_tile_rows(rows_per_cta);
+
+    static int configured_device = -1;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    if (configured_device != dev) {
+        cudaError_t e = cudaFuncSetAttribute(head_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+        if (e != cudaSuccess) return cuda_fail(e);
+        configured_device = dev;
+    }
+
+    CUtensorMap tmW;
+    r = make_map(&tmW, c.W, c.Vt, c.d, NT);
+    if (r != VT_OK) return r;
+
+    for (int m0 = 0; m0 < c.M; m0 += 128) {
+        const int mc = std::min(128, c.M - m0);
+        CUtensorMap tmH;
+        r = make_map(&tmH, c.h, c.M, c.d, mc);
+        if (r != VT_OK) return r;
+
+        MmaParams p{};
+        p.out = c.out;
+        p.m_begin = m0;
+        p.m_count = mc;
+        p.d = c.d;
+        p.NT = NT;
+        p.nk = (c.d + kBoxK - 1) / kBoxK;
+        p.a_tx = (uint32_t)mc * 128u;
+        p.b_tx = (uint32_t)NT * 128u;
+        p.stage_bytes = kABytes + (((uint32_t)NT * 128u + 1023u) & ~1023u);
+        // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
+        p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const size_t list_bytes = (size_t)c.out.k * 128 * 8;
+        const size_t bar_bytes = (size_t)(2 * 8 + 5) * 8 + 16;          // sized for the largest stage count
+        const size_t merge_bytes = (size_t)grid * (c.out.k + 1) * 8;
+        const size_t avail = (size_t)kMaxDynSmem - 1024 - list_bytes - bar_bytes - 256;
+        int S = (int)std::min<size_t>(8, avail / p.stage_bytes);
+        if (S < 2) return VT_ERR_UNSUPPORTED;
+        size_t ring = (size_t)S * p.stage_bytes;
+        if (ring < merge_bytes) return VT_ERR_UNSUPPORTED;              // cannot happen with S >= 2 (>= 36 KB)
+        p.n_stages = S;
+        p.list_off = (uint32_t)ring;
+        p.bar_off = (uint32_t)((ring + list_bytes + 127) & ~(size_t)127);
+        p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
+
+        head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmH, p);
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return VT_OK;
+}
+
 }  // namespace vt
