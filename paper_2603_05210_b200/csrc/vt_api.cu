@@ -47,6 +47,10 @@ static vt_status check_head_args(const void* h, const void* W, const int32_t* d2
     return VT_OK;
 }
 
+// Draft rows up to which the last head CTA merges the per-CTA records itself (one row per warp);
+// beyond that a separate merge kernel spreads the rows over many SMs.
+constexpr int kFusedMergeMaxM = 16;
+
 static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, float* lp, int32_t* did, float* lse,
                         float* logits, void* ws) {
     HeadOut o{};
@@ -58,24 +62,34 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
     o.logits = logits;
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
     o.hdr = reinterpret_cast<WsHeader*>(base);
-    o.keys = reinterpret_cast<unsigned long long*>(base + kHeaderBytes);
-    o.ms = reinterpret_cast<float2*>(base + kHeaderBytes + ws_keys_bytes(M, k));
+    o.recs = reinterpret_cast<unsigned long long*>(base + kHeaderBytes);
     o.M = M;
     o.k = k;
     o.Vt = Vt;
+    o.fused_merge = M <= kFusedMergeMaxM;
     return o;
 }
 
 // M at or below which the CUDA-core GEMV is used when both paths can run the shape.
-constexpr int kGemvMaxM = 4;
+constexpr int kAutoGemvMaxM = 2;
 
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
-    if (path == VT_PATH_GEMV) return launch_head_gemv(c, st);
-    if (path == VT_PATH_MMA) return launch_head_mma(c, st);
-    if (path != VT_PATH_AUTO) return VT_ERR_SHAPE;
-    if (c.M <= kGemvMaxM && gemv_supports(c.d)) return launch_head_gemv(c, st);
-    vt_status r = launch_head_mma(c, st);
-    if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st);
+    int grid = 0;
+    vt_status r;
+    if (path == VT_PATH_GEMV) {
+        r = launch_head_gemv(c, st, &grid);
+    } else if (path == VT_PATH_MMA) {
+        r = launch_head_mma(c, st, &grid);
+    } else if (path != VT_PATH_AUTO) {
+        return VT_ERR_SHAPE;
+    } else if (c.M <= kAutoGemvMaxM && gemv_supports(c.d)) {
+        r = launch_head_gemv(c, st, &grid);
+    } else {
+        r = launch_head_mma(c, st, &grid);
+        if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st, &grid);
+    }
+    if (r != VT_OK) return r;
+    if (!c.out.fused_merge) r = launch_merge(c.out, grid, st);
     return r;
 }
 

@@ -12,9 +12,11 @@ namespace vt {
 
 // ------------------------------------------------------------------------------------------
 // Workspace of a draft-head call:
-//   [0, 256)                       WsHeader
-//   keys  [kMaxParts][M][k] u64    per-CTA partial top-k lists (sortable keys, descending)
-//   ms    [kMaxParts][M] float2    per-CTA (running max, sum of exp(x - max))
+//   [0, 256)                          WsHeader
+//   recs [kMaxParts][M][KS] u64       per-CTA partial results, one record per (CTA, draft row):
+//                                     slots 0..k-1  top-k list as sortable keys, descending, 0-padded
+//                                     slot  k       (running max, sum of exp(x - max)) as two floats
+//                                     KS = k + 1 rounded up to even, so every record is 16-byte aligned
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxParts = 256;             // upper bound on CTAs that contribute partials
 constexpr size_t kHeaderBytes = 256;
@@ -28,24 +30,23 @@ static_assert(sizeof(WsHeader) == kHeaderBytes, "header is one 256-byte line");
 
 constexpr unsigned int kStatusTimeout = 1u;
 
-__host__ __device__ inline size_t ws_keys_bytes(int M, int k) { return (size_t)kMaxParts * M * k * 8; }
-__host__ __device__ inline size_t ws_ms_bytes(int M) { return (size_t)kMaxParts * M * 8; }
+__host__ __device__ inline int ws_slots(int k) { return (k + 2) & ~1; }
 __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
-    size_t b = kHeaderBytes + ws_keys_bytes(M, k) + ws_ms_bytes(M);
+    size_t b = kHeaderBytes + (size_t)kMaxParts * M * ws_slots(k) * 8;
     return (b + 255) & ~(size_t)255;
 }
 
 struct HeadOut {
-    const int32_t* d2t;
+    const int32_t* d2t;   // null: report draft indices as target ids
     int32_t* target_ids;
     float* logprobs;
     int32_t* draft_ids;   // may be null
     float* lse;           // may be null
     float* logits;        // debug: [M, Vt] fp32, null on the fast path
     WsHeader* hdr;
-    unsigned long long* keys;
-    float2* ms;
+    unsigned long long* recs;
     int M, k, Vt;
+    int fused_merge;      // 1: the last CTA to publish merges; 0: a merge kernel follows
 };
 
 #ifdef __CUDACC__
@@ -68,8 +69,8 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+__device__ __forceinline__ void fence_proxy_async() {      // generic <-> async proxy, all state spaces
+    asm volatile("fence.proxy.async;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -147,14 +148,6 @@ __device__ __forceinline__ void lse_update(float& mx, float& s, float x) {
     }
 }
 
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long w = __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        v = w > v ? w : v;
-    }
-    return v;
-}
 __device__ __forceinline__ float warp_max_f32(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
@@ -166,54 +159,79 @@ __device__ __forceinline__ float warp_sum_f32(float v) {
     return v;
 }
 
+__device__ __forceinline__ unsigned long long pack_ms(float mx, float s) {
+    return ((unsigned long long)__float_as_uint(s) << 32) | (unsigned long long)__float_as_uint(mx);
+}
+__device__ __forceinline__ float2 unpack_ms(unsigned long long v) {
+    return make_float2(__uint_as_float((uint32_t)v), __uint_as_float((uint32_t)(v >> 32)));
+}
+
+// Warp-wide maximum of 64-bit keys with two 32-bit redux operations.
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long v) {
+    const uint32_t hi = (uint32_t)(v >> 32), lo = (uint32_t)v;
+    const uint32_t mhi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    const uint32_t mlo = __reduce_max_sync(0xFFFFFFFFu, hi == mhi ? lo : 0u);
+    return ((unsigned long long)mhi << 32) | mlo;
+}
+
 // ------------------------------------------------------------------------------------------
-// Cross-CTA merge of one draft row by one warp.
-//   P partial lists (descending, k keys each, 0-padded) and
-//   P pairs (mx_p, s_p); both already staged in shared memory: stage[p * k + j], stage_ms[p].
-// Writes the row's k winners in descending key order with their log-probs and target ids.
+// Merge of P partial results of one draft row by one warp.  Partial p is a record in shared memory
+// at rec[p * stride]: k keys in descending order (0-padded), then (mx_p, s_p) in slot k.
+//   lse = mx + log sum_p s_p * exp(mx_p - mx),  mx = max_p mx_p
+// Every list is sorted, so a list's best remaining candidate is its head; lane L owns lists
+// L, L+32, ... and k rounds of a warp-wide maximum pick the winners in order.  Keys are unique
+// across lists (they carry distinct vocabulary rows), so exactly one head matches each round.
+// emit(j, key) is called by every lane with the round's winner (key 0: no candidate left).
 // ------------------------------------------------------------------------------------------
 constexpr int kMergeSlots = kMaxParts / 32;
 
-__device__ inline void merge_row(const HeadOut& o, int P, int m, const unsigned long long* stage,
-                                 const float2* stage_ms) {
+template <class Emit>
+__device__ __forceinline__ void warp_merge_lists(const unsigned long long* rec, int stride, int P, int k, Emit emit) {
     const int lane = threadIdx.x & 31;
-    const int k = o.k;
-
-    // log-sum-exp over the partials: lse = mx + log sum_p s_p * exp(mx_p - mx)
-    float mx = -INFINITY;
-    for (int p = lane; p < P; p += 32) mx = fmaxf(mx, stage_ms[p].x);
-    mx = warp_max_f32(mx);
-    float s = 0.0f;
-    for (int p = lane; p < P; p += 32) {
-        const float2 v = stage_ms[p];
-        if (v.y > 0.0f) s += v.y * __expf(v.x - mx);
-    }
-    s = warp_sum_f32(s);
-    const float lse = mx + logf(s);
-
-    // lane owns lists lane, lane+32, ...; every list is sorted, so its best is its head
     int head[kMergeSlots];
     unsigned long long hk[kMergeSlots];
 #pragma unroll
     for (int q = 0; q < kMergeSlots; ++q) {
         const int p = lane + 32 * q;
         head[q] = 0;
-        hk[q] = (p < P) ? stage[p * k] : 0ull;
+        hk[q] = (p < P) ? rec[(size_t)p * stride] : 0ull;
     }
     for (int j = 0; j < k; ++j) {
         unsigned long long best = 0ull;
 #pragma unroll
         for (int q = 0; q < kMergeSlots; ++q) best = hk[q] > best ? hk[q] : best;
-        best = warp_max_u64(best);
-        // keys are unique across lists (disjoint vocabulary rows), so exactly one head matches
+        best = warp_max_key(best);
 #pragma unroll
         for (int q = 0; q < kMergeSlots; ++q) {
             if (best != 0ull && hk[q] == best) {
-                const int p = lane + 32 * q;
                 ++head[q];
-                hk[q] = head[q] < k ? stage[p * k + head[q]] : 0ull;
+                hk[q] = head[q] < k ? rec[(size_t)(lane + 32 * q) * stride + head[q]] : 0ull;
             }
         }
+        emit(j, best);
+    }
+}
+
+__device__ __forceinline__ float2 warp_merge_ms(const unsigned long long* rec, int stride, int P, int k) {
+    const int lane = threadIdx.x & 31;
+    float mx = -INFINITY;
+    for (int p = lane; p < P; p += 32) mx = fmaxf(mx, unpack_ms(rec[(size_t)p * stride + k]).x);
+    mx = warp_max_f32(mx);
+    float s = 0.0f;
+    for (int p = lane; p < P; p += 32) {
+        const float2 v = unpack_ms(rec[(size_t)p * stride + k]);
+        if (v.y > 0.0f) s += v.y * __expf(v.x - mx);
+    }
+    return make_float2(mx, warp_sum_f32(s));
+}
+
+// Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
+__device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride) {
+    const int lane = threadIdx.x & 31;
+    const int k = o.k;
+    const float2 ms = warp_merge_ms(rec, stride, P, k);
+    const float lse = ms.x + logf(ms.y);
+    warp_merge_lists(rec, stride, P, k, [&](int j, unsigned long long best) {
         if (lane == 0) {
             const size_t out = (size_t)m * k + j;
             if (best != 0ull) {
@@ -227,14 +245,15 @@ __device__ inline void merge_row(const HeadOut& o, int P, int m, const unsigned 
                 if (o.draft_ids) o.draft_ids[out] = -1;
             }
         }
-    }
+    });
     if (lane == 0 && o.lse) o.lse[m] = lse;
 }
 
-// Publishes this CTA's partials (already written to global memory by the calling threads) and
+// Publishes this CTA's records (already written to global memory by the calling threads) and
 // returns true in every thread of the last CTA to arrive.  Must be called by all threads.
 __device__ inline bool publish_and_check_last(WsHeader* hdr, int* smem_flag) {
     __threadfence();
+    fence_proxy_async();          // the merging CTA reads the records with bulk copies (async proxy)
     __syncthreads();
     if (threadIdx.x == 0) {
         const unsigned int t = atomicAdd(&hdr->ticket, 1u);
@@ -245,53 +264,42 @@ __device__ inline bool publish_and_check_last(WsHeader* hdr, int* smem_flag) {
     return *smem_flag != 0;
 }
 
-// Last CTA: merges draft rows [m_begin, m_begin + m_count).  All threads first copy the partials of
-// a batch of rows from L2 into shared memory (independent loads, a few per thread), then each warp
-// merges one row at a time out of shared memory.  `stage_base` is shared memory the CTA no longer
-// uses; the host sizes it to hold at least one row: P * (k + 1) * 8 bytes.
+// Merges draft rows [m_begin, m_begin + m_count) from the records of P CTAs.  The records of a batch
+// of rows are brought into shared memory with one bulk copy per CTA record block (P copies in
+// flight at once: one L2 round trip per batch), then each warp merges one row at a time.
+//   stage_base/stage_bytes: shared memory the CTA no longer uses, 16-byte aligned, at least
+//                           P * (KS * 8 + 16) bytes;  bar: an initialised mbarrier (count 1), phase 0.
+// Must be called by all threads of the CTA.
 __device__ inline void merge_rows(const HeadOut& o, int P, int m_begin, int m_count,
-                                  unsigned char* stage_base, size_t stage_bytes) {
+                                  unsigned char* stage_base, size_t stage_bytes, uint32_t bar) {
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    const int k = o.k, M = o.M;
-    const size_t per_row = (size_t)P * (k + 1) * 8;
-    int batch = (int)(stage_bytes / per_row);
-    if (batch < 1) batch = 1;
+    const int KS = ws_slots(o.k), M = o.M;
+    int batch = (int)((stage_bytes / P - 16) / ((size_t)KS * 8));
+    const int tx_cap = (int)(((1u << 20) - 16) / ((size_t)P * KS * 8));     // mbarrier byte-count limit
+    if (batch > tx_cap) batch = tx_cap;
     if (batch > m_count) batch = m_count;
-    unsigned long long* skeys = reinterpret_cast<unsigned long long*>(stage_base);
-    float2* sms = reinterpret_cast<float2*>(stage_base + (size_t)batch * P * k * 8);
-    const int Pk = P * k;
-    for (int b0 = 0; b0 < m_count; b0 += batch) {
+    if (batch < 1) batch = 1;
+    unsigned long long* stage = reinterpret_cast<unsigned long long*>(stage_base);
+    fence_proxy_async();          // shared memory last touched by ordinary loads/stores is reused by bulk copies
+    __syncthreads();
+    uint32_t phase = 0;
+    for (int b0 = 0; b0 < m_count; b0 += batch, phase ^= 1u) {
         const int nb = min(batch, m_count - b0);
-        const int total = nb * Pk;
-        constexpr int U = 4;
-        for (int e0 = threadIdx.x; e0 < total; e0 += blockDim.x * U) {
-            unsigned long long v[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int e = e0 + u * blockDim.x;
-                if (e < total) {
-                    const int r = e / Pk, rem = e - r * Pk;
-                    const int p = rem / k, j = rem - p * k;
-                    v[u] = __ldcg(&o.keys[((size_t)p * M + (m_begin + b0 + r)) * k + j]);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int e = e0 + u * blockDim.x;
-                if (e < total) skeys[e] = v[u];
-            }
-        }
-        for (int e = threadIdx.x; e < nb * P; e += blockDim.x) {
-            const int r = e / P, p = e - r * P;
-            sms[e] = __ldcg(&o.ms[(size_t)p * M + (m_begin + b0 + r)]);
-        }
+        int stride = nb * KS;                                  // u64 units between CTA record blocks
+        if (((stride >> 1) & 1) == 0) stride += 2;             // odd multiple of 16 bytes: at most 2-way bank conflicts
+        const uint32_t bytes = (uint32_t)nb * KS * 8;
+        if (threadIdx.x == 0) mbar_arrive_expect_tx(bar, bytes * (uint32_t)P);
         __syncthreads();
-        for (int r = warp; r < nb; r += nwarps)
-            merge_row(o, P, m_begin + b0 + r, skeys + (size_t)r * Pk, sms + (size_t)r * P);
+        for (int p = threadIdx.x; p < P; p += blockDim.x)
+            bulk_g2s(smem_u32(stage + (size_t)p * stride), o.recs + ((size_t)p * M + m_begin + b0) * KS, bytes, bar);
+        if (!mbar_wait(bar, phase)) {
+            atomicOr(&o.hdr->status, kStatusTimeout);
+            break;
+        }
+        for (int r = warp; r < nb; r += nwarps) merge_row_final(o, P, m_begin + b0 + r, stage + (size_t)r * KS, stride);
         __syncthreads();
     }
-    if (threadIdx.x == 0) o.hdr->ticket = 0u;   // ready for the next call on this stream
 }
 #endif  // __CUDACC__
 

@@ -2,32 +2,41 @@
 //
 //   x[m, i] = sum_j h[m, j] * W_trim[i, j]          (the d -> k linear head, 2*d*k FLOPs per row)
 //
-// One persistent CTA per SM owns a contiguous range of vocabulary rows.  A producer thread
-// streams that range through a ring of shared-memory stages with 1-D bulk copies (whole rows are
-// contiguous in W_trim), consumer warps hold their column slice of h in registers, multiply with
-// packed fp32x2 FMAs and fold the per-lane partial sums with a transposing shuffle reduction, and
-// one epilogue warp finishes each logit, keeps a running (max, sum-exp) and a top-k list per draft
-// row, and never writes a logit to memory.  The last CTA to publish its partials merges them.
+// One persistent CTA per SM owns a contiguous range of vocabulary rows.  A producer thread streams
+// that range through a ring of shared-memory stages with 1-D bulk copies (whole rows are contiguous
+// in W_trim).  Each stage holds a few complete rows and is consumed by ONE warp: its lanes stride
+// over the row in 16-byte chunks, multiply with the bf16 hidden states kept in shared memory using
+// packed fp32x2 FMAs, and fold the lane partials with a transposing shuffle reduction.  The lane
+// that ends up with a logit keeps that (row slot, draft row)'s running (max, sum-exp) and top-k
+// list, so no logit is written to memory and no warp waits for another.  When the range is done
+// the CTA folds its warps' lists into one record per draft row; the last CTA to publish merges all
+// CTAs' records (or a merge kernel does, for many draft rows).
+//
+// The FP32 pipe bounds this path: every weight costs M fused multiply-adds, which the CUDA cores
+// keep up with only for M <= 4; larger M belongs to the tensor-core path.
 #include "vt_common.cuh"
 #include "vt_launch.h"
 
 namespace vt {
 
+constexpr int kGemvWarps = 16;                 // 1 producer + 15 consumers
+constexpr int kGemvConsumers = kGemvWarps - 1;
+constexpr int kGemvThreads = kGemvWarps * 32;
+constexpr int kGemvR = 2;                      // vocabulary rows a warp accumulates together
+constexpr int kGemvMaxM = 4;                   // draft rows per pass
+
 struct GemvParams {
     const uint16_t* h;       // [M, d] bf16 (already offset to the first row of this pass)
     const uint16_t* W;       // [Vt, d] bf16
     HeadOut out;
-    int m_begin;             // first draft row of this pass (index into out.*)
-    int m_count;             // rows in this pass, <= MP
+    int m_begin, m_count;    // draft rows of this pass
     int d;
-    int rows_per_stage;
-    int n_stages;
-    int ncw;                 // consumer warps
+    int rows_per_stage;      // multiple of kGemvR
+    int n_stages;            // multiple of n_cons, so a stage is always consumed by the same warp
+    int n_cons;              // consumer warps that take tiles (<= kGemvConsumers)
     uint32_t stage_bytes;
-    uint32_t red_off, list_off, bar_off, total_smem;
+    uint32_t h_off, list_off, bar_off, total_smem;
 };
-
-__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 
 // Folds NV per-lane values over the 32 lanes of a warp with NV-1 + log2(32/NV) shuffles.
 // Afterwards every lane holds the warp total of value index (lane >> (5 - log2 NV)).
@@ -52,13 +61,17 @@ __device__ __forceinline__ void fold_step(float* v, int lane) {
 template <int N> struct Log2 { static constexpr int value = 1 + Log2<N / 2>::value; };
 template <> struct Log2<1> { static constexpr int value = 0; };
 
-// MP: draft rows per pass padded to a power of two; CPT: 16-byte column chunks per consumer thread;
-// R: vocabulary rows accumulated together before a fold; MAXT: launch bound.
-template <int MP, int CPT, int R, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1) head_gemv_kernel(const GemvParams p) {
+__device__ __forceinline__ float2 bf16x2_to_f32x2(uint32_t w) {
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+}
+
+// MP: draft rows per pass padded to a power of two.
+template <int MP>
+__global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int NV = R * MP;
-    static_assert(NV <= 32 && (NV & (NV - 1)) == 0, "fold width");
+    constexpr int R = kGemvR;
+    constexpr int NV = R * MP;                         // logits a warp finishes per fold
+    constexpr int SHIFT = 5 - Log2<NV>::value;         // owner lane of value index i is i << SHIFT
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
@@ -66,39 +79,42 @@ __global__ void __launch_bounds__(MAXT, 1) head_gemv_kernel(const GemvParams p) 
     const int row_begin = (int)((long long)cta * Vt / G);
     const int row_end = (int)((long long)(cta + 1) * Vt / G);
     const int nrows = row_end - row_begin;
-    const int SR = p.rows_per_stage, S = p.n_stages, ncw = p.ncw;
+    const int SR = p.rows_per_stage, S = p.n_stages;
     const int ntiles = (nrows + SR - 1) / SR;
+    const int KS = ws_slots(k);
 
-    float* red = reinterpret_cast<float*>(smem + p.red_off);                       // [2][SR][ncw][MP]
-    unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [k][MP]
+    unsigned char* hs = smem + p.h_off;                                                      // [MP][d] bf16
+    unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [consumer][NV][KS]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
-    // bars: full[S], empty[S], red_full[2], red_empty[2]; then two ints: abort flag, last flag
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * S;
-    const uint32_t bar_rfull = bar_empty + 8u * S, bar_rempty = bar_rfull + 16u;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * S + 4);
+    // bars: full[S], empty[S], merge; then two ints: abort flag, last flag
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * S, bar_merge = bar_empty + 8u * S;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * S + 1);
     int* last_flag = const_cast<int*>(abort_flag) + 1;
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8u * s, 1);
-            mbar_init(bar_empty + 8u * s, ncw);
+            mbar_init(bar_empty + 8u * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_rfull + 8u * b, ncw);
-            mbar_init(bar_rempty + 8u * b, 1);
-        }
+        mbar_init(bar_merge, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
-    for (int i = tid; i < k * MP; i += blockDim.x) lists[i] = 0ull;
+    for (int i = tid; i < kGemvConsumers * NV * KS; i += blockDim.x) lists[i] = 0ull;
+    {   // hidden states of this pass; pad rows (m >= m_count) repeat the last real row and are never read out
+        const int nchunks = d >> 3;
+        for (int i = tid; i < MP * nchunks; i += blockDim.x) {
+            const int m = i / nchunks, c = i - m * nchunks;
+            const int msrc = min(m, p.m_count - 1);
+            reinterpret_cast<uint4*>(hs)[i] = __ldg(reinterpret_cast<const uint4*>(p.h + (size_t)msrc * d) + c);
+        }
+    }
     __syncthreads();
 
     auto fail = [&]() {
         *abort_flag = 1;
         atomicOr(&p.out.hdr->status, kStatusTimeout);
     };
-
-    float mx = -INFINITY, ssum = 0.0f;     // epilogue state of lane m < m_count
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -120,67 +136,22 @@ __global__ void __launch_bounds__(MAXT, 1) head_gemv_kernel(const GemvParams p) 
                     (void)mbar_wait(bar_full + 8u * (t % S), (uint32_t)(t / S) & 1u);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ epilogue warp
-        constexpr int NPARTS = 32 / MP;
-        const int m = lane % MP, part = lane / MP;
-        const bool owner = (part == 0) && (m < p.m_count);
-        unsigned long long thr = 0ull;
-        for (int t = 0; t < ntiles; ++t) {
-            const int buf = t & 1;
-            if (!mbar_wait(bar_rfull + 8u * buf, (uint32_t)(t >> 1) & 1u)) { fail(); break; }
-            if (*abort_flag) break;
-            const int rows = min(SR, nrows - t * SR);
-            for (int r = 0; r < rows; ++r) {
-                const float* src = red + ((size_t)(buf * SR + r) * ncw) * MP + m;
-                float x = 0.0f;
-                for (int cw = part; cw < ncw; cw += NPARTS) x += src[cw * MP];
-#pragma unroll
-                for (int o = MP; o < 32; o <<= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-                if (owner) {
-                    const int row = row_begin + t * SR + r;
-                    lse_update(mx, ssum, x);
-                    const unsigned long long key = make_key(x, row);
-                    if (key > thr) thr = list_insert(lists + m, MP, k, key);
-                    if (p.out.logits) p.out.logits[(size_t)(p.m_begin + m) * Vt + row] = x;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_rempty + 8u * buf);
-        }
-        __syncwarp();
-        if (owner) {
-            const size_t slot = (size_t)cta * M + p.m_begin + m;
-            for (int j = 0; j < k; ++j) p.out.keys[slot * k + j] = lists[j * MP + m];
-            p.out.ms[slot] = make_float2(mx, ssum);
-        }
-    } else if (warp - 2 < ncw) {
-        // ------------------------------------------------------------------ consumers
-        const int cw = warp - 2;
+    } else {
+        // ------------------------------------------------------------------ consumers: one warp per stage
+        const int cw = warp - 1;
         const int nchunks = d >> 3;
-        float2 hp[CPT][4][MP];
-        int chunk[CPT];
-#pragma unroll
-        for (int q = 0; q < CPT; ++q) {
-            chunk[q] = cw * 32 + lane + q * ncw * 32;
-            const bool valid = chunk[q] < nchunks;
-#pragma unroll
-            for (int m = 0; m < MP; ++m) {
-                uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                if (valid && m < p.m_count)
-                    w = __ldg(reinterpret_cast<const uint4*>(p.h + (size_t)m * d + (size_t)chunk[q] * 8));
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj)
-                    hp[q][jj][m] = make_float2(__uint_as_float(ww[jj] << 16), __uint_as_float(ww[jj] & 0xFFFF0000u));
-            }
-            if (!valid) chunk[q] = -1;
-        }
-        constexpr int SHIFT = 5 - Log2<NV>::value;
-        for (int t = 0; t < ntiles; ++t) {
-            const int s = t % S, buf = t & 1;
+        const int my_idx = lane >> SHIFT;                       // value index this lane ends up holding
+        const bool owner = (lane & ((1 << SHIFT) - 1)) == 0;
+        const int my_r = my_idx / MP, my_m = my_idx % MP;
+        const bool live = owner && my_m < p.m_count;
+        unsigned long long* my_list = lists + (size_t)(cw * NV + my_idx) * KS;
+        float mx = -INFINITY, ssum = 0.0f, thr_x = -INFINITY;
+        int filled = 0;
+        // Tile t lives in stage t % S and belongs to warp t % n_cons.  S is a multiple of n_cons, so one warp sees
+        // every phase of the stages it uses, in order (a parity wait may lag its barrier by one phase at most).
+        for (int t = cw; t < ntiles && cw < p.n_cons; t += p.n_cons) {
+            const int s = t % S;
             if (!mbar_wait(bar_full + 8u * s, (uint32_t)(t / S) & 1u)) { fail(); break; }
-            if (t >= 2 && !mbar_wait(bar_rempty + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
             if (*abort_flag) break;
             const int rows = min(SR, nrows - t * SR);
             const unsigned char* stage = smem + (size_t)s * p.stage_bytes;
@@ -190,23 +161,25 @@ __global__ void __launch_bounds__(MAXT, 1) head_gemv_kernel(const GemvParams p) 
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int m = 0; m < MP; ++m) acc[r][m] = make_float2(0.0f, 0.0f);
+                // a row slot past the tile's last row re-reads the last row; its result is dropped below
+                const unsigned char* wrow[R];
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (g0 + r < rows) {
+                for (int r = 0; r < R; ++r) wrow[r] = stage + (size_t)min(g0 + r, rows - 1) * d * 2;
+                for (int c = lane; c < nchunks; c += 32) {
+                    uint4 w[R];
 #pragma unroll
-                        for (int q = 0; q < CPT; ++q) {
-                            if (chunk[q] >= 0) {
-                                const uint4 w = *reinterpret_cast<const uint4*>(
-                                    stage + ((size_t)(g0 + r) * d + (size_t)chunk[q] * 8) * 2);
-                                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                    for (int r = 0; r < R; ++r) w[r] = *reinterpret_cast<const uint4*>(wrow[r] + (size_t)c * 16);
 #pragma unroll
-                                for (int jj = 0; jj < 4; ++jj) {
-                                    const float2 wp = make_float2(__uint_as_float(ww[jj] << 16),
-                                                                  __uint_as_float(ww[jj] & 0xFFFF0000u));
+                    for (int m = 0; m < MP; ++m) {
+                        const uint4 hv = *reinterpret_cast<const uint4*>(hs + ((size_t)m * d + (size_t)c * 8) * 2);
+                        const float2 h0 = bf16x2_to_f32x2(hv.x), h1 = bf16x2_to_f32x2(hv.y);
+                        const float2 h2 = bf16x2_to_f32x2(hv.z), h3 = bf16x2_to_f32x2(hv.w);
 #pragma unroll
-                                    for (int m = 0; m < MP; ++m) acc[r][m] = ffma2(wp, hp[q][jj][m], acc[r][m]);
-                                }
-                            }
+                        for (int r = 0; r < R; ++r) {
+                            acc[r][m] = __ffma2_rn(bf16x2_to_f32x2(w[r].x), h0, acc[r][m]);
+                            acc[r][m] = __ffma2_rn(bf16x2_to_f32x2(w[r].y), h1, acc[r][m]);
+                            acc[r][m] = __ffma2_rn(bf16x2_to_f32x2(w[r].z), h2, acc[r][m]);
+                            acc[r][m] = __ffma2_rn(bf16x2_to_f32x2(w[r].w), h3, acc[r][m]);
                         }
                     }
                 }
@@ -216,31 +189,54 @@ __global__ void __launch_bounds__(MAXT, 1) head_gemv_kernel(const GemvParams p) 
 #pragma unroll
                     for (int m = 0; m < MP; ++m) v[r * MP + m] = acc[r][m].x + acc[r][m].y;
                 fold_step<NV, 16>(v, lane);
-                if ((lane & ((1 << SHIFT) - 1)) == 0) {
-                    const int idx = lane >> SHIFT;
-                    const int r = idx / MP, m = idx % MP;
-                    if (g0 + r < rows) red[((size_t)(buf * SR + g0 + r) * ncw + cw) * MP + m] = v[0];
+                if (live && g0 + my_r < rows) {
+                    const float x = v[0];
+                    const int row = row_begin + t * SR + g0 + my_r;
+                    lse_update(mx, ssum, x);
+                    if (x > thr_x || filled < k) {     // rows reach this lane in ascending order: ties lose
+                        const unsigned long long kth = list_insert(my_list, 1, k, make_key(x, row));
+                        if (filled < k) ++filled;
+                        if (filled == k) thr_x = key_logit(kth);
+                    }
+                    if (p.out.logits) p.out.logits[(size_t)(p.m_begin + my_m) * Vt + row] = x;
                 }
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar_empty + 8u * s);
-                mbar_arrive(bar_rfull + 8u * buf);
-            }
+            if (lane == 0) mbar_arrive(bar_empty + 8u * s);
         }
+        if (owner) my_list[k] = pack_ms(mx, ssum);
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------------- fold the CTA's lists: one warp per draft row
+    if (warp < p.m_count) {
+        // lists of draft row `warp`: index (cw * NV + r * MP + warp), i.e. P1 = consumers * R lists, KS apart * MP
+        const int m = warp;
+        const int P1 = kGemvConsumers * R;
+        const unsigned long long* rec0 = lists + (size_t)m * KS;
+        const int stride = MP * KS;
+        const float2 ms = warp_merge_ms(rec0, stride, P1, k);
+        unsigned long long* dst = p.out.recs + ((size_t)cta * M + p.m_begin + m) * KS;
+        warp_merge_lists(rec0, stride, P1, k, [&](int j, unsigned long long best) {
+            if (lane == 0) dst[j] = best;
+        });
+        if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
     }
 
-    // ---------------------------------------------------------------------- publish + merge
-    if (publish_and_check_last(p.out.hdr, last_flag))
-        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.bar_off);   // ring, red and lists are free now
+    // ---------------------------------------------------------------------- publish (+ merge)
+    if (!p.out.fused_merge) return;
+    if (publish_and_check_last(p.out.hdr, last_flag)) {
+        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.bar_off, bar_merge);   // ring, h and lists are free now
+        if (tid == 0) p.out.hdr->ticket = 0u;                                      // ready for the next call
+    }
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
-template <int MP, int CPT, int R, int MAXT>
-static vt_status launch_one(const GemvParams& p, int grid, int threads, cudaStream_t st) {
-    auto kern = head_gemv_kernel<MP, CPT, R, MAXT>;
+template <int MP>
+static vt_status launch_one(const GemvParams& p, int grid, cudaStream_t st) {
+    auto kern = head_gemv_kernel<MP>;
     static int configured_device = -1;   // per instantiation
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
@@ -249,7 +245,7 @@ static vt_status launch_one(const GemvParams& p, int grid, int threads, cudaStre
         if (e != cudaSuccess) return cuda_fail(e);
         configured_device = dev;
     }
-    kern<<<grid, threads, p.total_smem, st>>>(p);
+    kern<<<grid, kGemvThreads, p.total_smem, st>>>(p);
     count_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
@@ -257,25 +253,18 @@ static vt_status launch_one(const GemvParams& p, int grid, int threads, cudaStre
 
 bool gemv_supports(int d) { return d >= 8 && d % 8 == 0 && d <= 8192; }
 
-vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st) {
+vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
     if (!gemv_supports(c.d)) return VT_ERR_UNSUPPORTED;
-    const int nchunks = c.d / 8;
     int sms = 0;
     vt_status rs = device_sm_count(&sms);
     if (rs != VT_OK) return rs;
-    const int grid = std::max(1, std::min(std::min(sms, kMaxParts), c.Vt));
+    const int grid = head_grid(sms, c.Vt);
+    *grid_out = grid;
+    const int KS = ws_slots(c.out.k);
 
-    for (int m0 = 0; m0 < c.M; m0 += 8) {
-        const int mc = std::min(8, c.M - m0);
-        const int MP = mc <= 1 ? 1 : mc <= 2 ? 2 : mc <= 4 ? 4 : 8;
-        // consumer warps and chunks per thread: MP = 8 keeps its h slice in 64 registers, so one chunk only
-        int cpt = 1, ncw = (nchunks + 31) / 32;
-        if (ncw > 16) {
-            if (MP == 8 || ncw > 20) { cpt = 2; ncw = (nchunks + 63) / 64; }
-        }
-        if (MP == 8 && cpt == 2) return VT_ERR_UNSUPPORTED;   // h slice would not fit the register file
-        const int R = (MP == 8) ? 2 : 4;
-        const int threads = (ncw + 2) * 32;
+    for (int m0 = 0; m0 < c.M; m0 += kGemvMaxM) {
+        const int mc = std::min(kGemvMaxM, c.M - m0);
+        const int MP = mc <= 1 ? 1 : mc <= 2 ? 2 : 4;
 
         GemvParams p{};
         p.h = reinterpret_cast<const uint16_t*>(c.h) + (size_t)m0 * c.d;
@@ -284,52 +273,32 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st) {
         p.m_begin = m0;
         p.m_count = mc;
         p.d = c.d;
-        p.ncw = ncw;
-        int sr = 32768 / (2 * c.d);
-        sr = std::max(R, std::min(16, sr) / R * R);
+        int sr = 16384 / (2 * c.d);
+        sr = std::max(kGemvR, std::min(16, sr) / kGemvR * kGemvR);
         p.rows_per_stage = sr;
         p.stage_bytes = (uint32_t)sr * c.d * 2;
-        const size_t red_bytes = (size_t)2 * sr * ncw * MP * 4;
-        const size_t list_bytes = (size_t)c.out.k * MP * 8;
-        const size_t bar_bytes = 0;   // sized below, needs n_stages
-        (void)bar_bytes;
-        const size_t merge_bytes = (size_t)grid * (c.out.k + 1) * 8;
-        // stages: as many as fit next to the small buffers, at most 8
-        int S = 8;
-        size_t ring, total;
-        for (;; --S) {
-            ring = (size_t)S * p.stage_bytes;
-            size_t off = (ring + 127) & ~(size_t)127;
-            p.red_off = (uint32_t)off;
-            off += (red_bytes + 127) & ~(size_t)127;
-            p.list_off = (uint32_t)off;
-            off += (list_bytes + 127) & ~(size_t)127;
-            if (off < merge_bytes) off = (merge_bytes + 127) & ~(size_t)127;   // merge staging reuses [0, bar_off)
-            p.bar_off = (uint32_t)off;
-            total = off + (size_t)(2 * S + 4) * 8 + 16;
-            if (total <= (size_t)kMaxDynSmem || S == 2) break;
-        }
-        if (total > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
+        const size_t h_bytes = ((size_t)MP * c.d * 2 + 127) & ~(size_t)127;
+        const size_t list_bytes = ((size_t)kGemvConsumers * kGemvR * MP * KS * 8 + 127) & ~(size_t)127;
+        const size_t merge_bytes = (size_t)grid * (KS * 8 + 16);
+        const size_t bar_bytes = (size_t)(2 * 32 + 1) * 8 + 16;
+        const size_t fixed = h_bytes + list_bytes + bar_bytes;
+        if (fixed + 2 * (size_t)p.stage_bytes > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
+        int S = (int)std::min<size_t>(32, ((size_t)kMaxDynSmem - fixed) / p.stage_bytes);
+        p.n_cons = std::min(kGemvConsumers, S);
+        S = S / p.n_cons * p.n_cons;
+        size_t off = (size_t)S * p.stage_bytes;
         p.n_stages = S;
-        p.total_smem = (uint32_t)total;
+        p.h_off = (uint32_t)off;
+        off += h_bytes;
+        p.list_off = (uint32_t)off;
+        off += list_bytes;
+        if (off < merge_bytes) off = (merge_bytes + 127) & ~(size_t)127;   // merge staging reuses [0, bar_off)
+        p.bar_off = (uint32_t)off;
+        p.total_smem = (uint32_t)(off + bar_bytes);
+        if (p.total_smem > (uint32_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
 
-        vt_status r = VT_ERR_UNSUPPORTED;
-#define VT_GEMV_CASE(MP_, CPT_, R_)                                                            \
-        if (MP == MP_ && cpt == CPT_) {                                                        \
-            r = (threads <= 576) ? launch_one<MP_, CPT_, R_, 576>(p, grid, threads, st)        \
-                                 : launch_one<MP_, CPT_, R_, 704>(p, grid, threads, st);       \
-        }
-        VT_GEMV_CASE(1, 1, 4)
-        VT_GEMV_CASE(2, 1, 4)
-        VT_GEMV_CASE(4, 1, 4)
-        VT_GEMV_CASE(1, 2, 4)
-        VT_GEMV_CASE(2, 2, 4)
-        VT_GEMV_CASE(4, 2, 4)
-#undef VT_GEMV_CASE
-        if (MP == 8 && cpt == 1) {
-            if (threads > 576) return VT_ERR_UNSUPPORTED;
-            r = launch_one<8, 1, 2, 576>(p, grid, threads, st);
-        }
+        vt_status r = MP == 1 ? launch_one<1>(p, grid, st) : MP == 2 ? launch_one<2>(p, grid, st)
+                                                                      : launch_one<4>(p, grid, st);
         if (r != VT_OK) return r;
     }
     return VT_OK;

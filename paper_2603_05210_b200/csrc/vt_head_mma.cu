@@ -20,9 +20,9 @@
 
 namespace vt {
 
-constexpr int kMmaThreads = 192;
+constexpr int kMmaThreads = 512;               // warps 0-3 epilogue, 4 TMA, 5 MMA; the rest only join the final merge
 constexpr int kBoxK = 64;                    // bf16 elements per k-step = one 128-byte swizzle row
-constexpr uint32_t kABytes = 128 * 128;      // A slot: 128 rows x 128 B (only the pass's rows are copied)
+constexpr int kMaxStages = 32;
 constexpr int kAccStride = 256;              // TMEM columns between the two accumulator buffers
 
 struct MmaParams {
@@ -33,6 +33,7 @@ struct MmaParams {
     int nk;                   // k-steps per tile
     int n_stages;
     uint32_t stage_bytes;     // A slot + B slot, multiple of 1024
+    uint32_t a_slot;          // bytes of the A slot: the pass's rows rounded up to whole 8-row groups
     uint32_t a_tx, b_tx;      // bytes each TMA box delivers
     uint32_t idesc;
     uint32_t list_off, bar_off, total_smem;   // offsets from the 1024-aligned base
@@ -102,7 +103,8 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
     const uint32_t bar_full = base + p.bar_off, bar_empty = bar_full + 8u * S;
     const uint32_t bar_accf = bar_empty + 8u * S, bar_acce = bar_accf + 16u, bar_drain = bar_acce + 16u;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 5);
+    const uint32_t bar_merge = bar_drain + 8u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_flag = const_cast<int*>(abort_flag) + 1;
 
@@ -117,10 +119,13 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             mbar_init(bar_acce + 8u * b, n_epi_warps);
         }
         mbar_init(bar_drain, 1);
+        mbar_init(bar_merge, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
     for (int i = tid; i < k * 128; i += blockDim.x) lists[i] = 0ull;
+    // The MMA always reads 128 A rows; rows past the pass's last row hold whatever follows the A slot in
+    // shared memory.  They only feed TMEM lanes that no thread reads, so they are left as they are.
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
@@ -150,7 +155,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                     const uint32_t a_dst = base + (uint32_t)s * p.stage_bytes;
                     mbar_arrive_expect_tx(bar_full + 8u * s, p.a_tx + p.b_tx);
                     tma_load_2d(a_dst, &tmH, ks * kBoxK, p.m_begin, bar_full + 8u * s);
-                    tma_load_2d(a_dst + kABytes, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
+                    tma_load_2d(a_dst + p.a_slot, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
                     issued = it + 1;
                 }
             }
@@ -175,7 +180,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = base + (uint32_t)s * p.stage_bytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + kABytes);
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + p.a_slot);
 #pragma unroll
                     for (int kk = 0; kk < kBoxK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
                         tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, p.idesc, (ks | kk) != 0);
@@ -246,19 +251,23 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
         }
         if (live) {
-            const size_t slot = (size_t)cta * M + p.m_begin + m_local;
-            for (int j = 0; j < k; ++j) p.out.keys[slot * k + j] = my_list[j * 128];
-            p.out.ms[slot] = make_float2(mx, ssum);
+            unsigned long long* rec = p.out.recs + ((size_t)cta * M + p.m_begin + m_local) * ws_slots(k);
+            for (int j = 0; j < k; ++j) rec[j] = my_list[j * 128];
+            rec[k] = pack_ms(mx, ssum);
         }
     }
 
     // ---------------------------------------------------------------------- publish + merge
     tc_fence_before();
-    const bool last = publish_and_check_last(p.out.hdr, last_flag);
+    __syncthreads();
     tc_fence_after();
     if (warp == 5)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
-    if (last) merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.list_off);   // the ring is free now
+    if (!p.out.fused_merge) return;
+    if (publish_and_check_last(p.out.hdr, last_flag)) {
+        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.list_off, bar_merge);   // the ring is free now
+        if (tid == 0) p.out.hdr->ticket = 0u;                                       // ready for the next call
+    }
 }
 
 // ------------------------------------------------------------------------------------------ host
@@ -310,11 +319,12 @@ static int choose_tile_rows(int rows_per_cta) {
     return best;
 }
 
-vt_status launch_head_mma(const HeadCall& c, cudaStream_t st) {
+vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     int sms = 0;
     vt_status r = device_sm_count(&sms);
     if (r != VT_OK) return r;
-    const int grid = std::max(1, std::min(std::min(sms, kMaxParts), (c.Vt + 15) / 16));
+    const int grid = head_grid(sms, c.Vt, 16);
+    *grid_out = grid;
     const int rows_per_cta = (c.Vt + grid - 1) / grid;
     const int NT = choose_tile_rows(rows_per_cta);
 
@@ -346,21 +356,26 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st) {
         p.nk = (c.d + kBoxK - 1) / kBoxK;
         p.a_tx = (uint32_t)mc * 128u;
         p.b_tx = (uint32_t)NT * 128u;
-        p.stage_bytes = kABytes + (((uint32_t)NT * 128u + 1023u) & ~1023u);
+        p.a_slot = (((uint32_t)mc * 128u) + 1023u) & ~1023u;
+        p.stage_bytes = p.a_slot + (((uint32_t)NT * 128u + 1023u) & ~1023u);
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         const size_t list_bytes = (size_t)c.out.k * 128 * 8;
-        const size_t bar_bytes = (size_t)(2 * 8 + 5) * 8 + 16;          // sized for the largest stage count
-        const size_t merge_bytes = (size_t)grid * (c.out.k + 1) * 8;
-        const size_t avail = (size_t)kMaxDynSmem - 1024 - list_bytes - bar_bytes - 256;
-        int S = (int)std::min<size_t>(8, avail / p.stage_bytes);
+        const size_t bar_bytes = (size_t)(2 * kMaxStages + 6) * 8 + 16;  // sized for the largest stage count
+        const size_t merge_bytes = (size_t)grid * (ws_slots(c.out.k) * 8 + 16);
+        // the MMA reads 128 A rows from the slot's start: keep 16 KB readable past the last stage's A slot
+        const size_t avail = (size_t)kMaxDynSmem - 1024 - list_bytes - bar_bytes - 256 - 16384;
+        int S = (int)std::min<size_t>(kMaxStages, avail / p.stage_bytes);
         if (S < 2) return VT_ERR_UNSUPPORTED;
         size_t ring = (size_t)S * p.stage_bytes;
-        if (ring < merge_bytes) return VT_ERR_UNSUPPORTED;              // cannot happen with S >= 2 (>= 36 KB)
+        if (ring < 16384 + (size_t)p.stage_bytes) ring = 16384 + p.stage_bytes;
+        if (ring < merge_bytes) ring = (merge_bytes + 1023) & ~(size_t)1023;
+        if (ring + list_bytes + bar_bytes + 1024 + 256 > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
         p.n_stages = S;
         p.list_off = (uint32_t)ring;
         p.bar_off = (uint32_t)((ring + list_bytes + 127) & ~(size_t)127);
-        p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
+        const size_t a_overread = (size_t)(S - 1) * p.stage_bytes + 16384;     // last A slot + 128 rows
+        p.total_smem = (uint32_t)(std::max<size_t>(p.bar_off + bar_bytes, a_overread) + 1024);
 
         head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmH, p);
         count_launch();

@@ -24,9 +24,17 @@ vt_status driver_fail(int cu_result);
 void count_launch();
 vt_status device_sm_count(int* sms);
 
+// Both head kernels split the vocabulary rows over `*grid` persistent CTAs (one per SM at most); the
+// merge needs to know how many CTAs wrote records.
+inline int head_grid(int sms, int Vt, int min_rows_per_cta = 1) {
+    const int by_rows = (Vt + min_rows_per_cta - 1) / min_rows_per_cta;
+    return std::max(1, std::min(std::min(sms, kMaxParts), by_rows));
+}
+
 bool gemv_supports(int d);
-vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st);
-vt_status launch_head_mma(const HeadCall& c, cudaStream_t st);
+vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid);
+vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid);
+vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st);
 
 vt_status launch_compact(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim,
                          void* W_trim, cudaStream_t st);

@@ -1,0 +1,46 @@
+// Stand-alone cross-CTA merge for calls with many draft rows: one CTA per group of rows, so the merge
+// of M rows runs on M / 8 SMs at once instead of on the last head CTA alone.
+#include "vt_common.cuh"
+#include "vt_launch.h"
+
+namespace vt {
+
+constexpr int kMergeThreads = 256;
+constexpr int kMergeRowsPerCta = kMergeThreads / 32;
+
+__global__ void __launch_bounds__(kMergeThreads) merge_kernel(const HeadOut o, int P, uint32_t stage_bytes) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const int m_begin = blockIdx.x * kMergeRowsPerCta;
+    const int m_count = min(kMergeRowsPerCta, o.M - m_begin);
+    merge_rows(o, P, m_begin, m_count, smem, stage_bytes, smem_u32(&bar));
+}
+
+vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st) {
+    const int KS = ws_slots(o.k);
+    const size_t one_row = (size_t)P * (KS * 8 + 16);
+    size_t want = (size_t)P * ((size_t)kMergeRowsPerCta * KS * 8 + 16);
+    const size_t cap = 160 * 1024;
+    if (want > cap) want = std::max(one_row, cap / one_row * one_row);
+    if (want > (size_t)kMaxDynSmem - 1024) return VT_ERR_UNSUPPORTED;
+    static int configured_device = -1;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    if (configured_device != dev) {
+        cudaError_t e = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem - 1024);
+        if (e != cudaSuccess) return cuda_fail(e);
+        configured_device = dev;
+    }
+    const int grid = (o.M + kMergeRowsPerCta - 1) / kMergeRowsPerCta;
+    merge_kernel<<<grid, kMergeThreads, want, st>>>(o, P, (uint32_t)want);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+}  // namespace vt
