@@ -181,35 +181,49 @@ __device__ __forceinline__ unsigned long long warp_max_key(unsigned long long v)
 // Every list is sorted, so a list's best remaining candidate is its head; lane L owns lists
 // L, L+32, ... and k rounds of a warp-wide maximum pick the winners in order.  Keys are unique
 // across lists (they carry distinct vocabulary rows), so exactly one head matches each round.
-// emit(j, key) is called by every lane with the round's winner (key 0: no candidate left).
 // ------------------------------------------------------------------------------------------
 constexpr int kMergeSlots = kMaxParts / 32;
 
-template <class Emit>
-__device__ __forceinline__ void warp_merge_lists(const unsigned long long* rec, int stride, int P, int k, Emit emit) {
+// SLOTS >= ceil(P / 32).  Returns this lane's share of the winners: winner j sits in lane j % 32,
+// element j / 32 of `mine` (k <= 64).
+template <int SLOTS>
+__device__ __forceinline__ void warp_merge_lists_n(const unsigned long long* rec, int stride, int P, int k,
+                                                   unsigned long long (&mine)[2]) {
     const int lane = threadIdx.x & 31;
-    int head[kMergeSlots];
-    unsigned long long hk[kMergeSlots];
+    int head[SLOTS];
+    unsigned long long hk[SLOTS];
+    unsigned long long local = 0ull;
 #pragma unroll
-    for (int q = 0; q < kMergeSlots; ++q) {
+    for (int q = 0; q < SLOTS; ++q) {
         const int p = lane + 32 * q;
         head[q] = 0;
         hk[q] = (p < P) ? rec[(size_t)p * stride] : 0ull;
+        local = hk[q] > local ? hk[q] : local;
     }
+    mine[0] = mine[1] = 0ull;
     for (int j = 0; j < k; ++j) {
-        unsigned long long best = 0ull;
+        const unsigned long long best = warp_max_key(local);
+        if (best != 0ull && local == best) {          // the one lane whose head won advances that list
+            local = 0ull;
 #pragma unroll
-        for (int q = 0; q < kMergeSlots; ++q) best = hk[q] > best ? hk[q] : best;
-        best = warp_max_key(best);
-#pragma unroll
-        for (int q = 0; q < kMergeSlots; ++q) {
-            if (best != 0ull && hk[q] == best) {
-                ++head[q];
-                hk[q] = head[q] < k ? rec[(size_t)(lane + 32 * q) * stride + head[q]] : 0ull;
+            for (int q = 0; q < SLOTS; ++q) {
+                if (hk[q] == best) {
+                    ++head[q];
+                    hk[q] = head[q] < k ? rec[(size_t)(lane + 32 * q) * stride + head[q]] : 0ull;
+                }
+                local = hk[q] > local ? hk[q] : local;
             }
         }
-        emit(j, best);
+        if ((j & 31) == lane) mine[j >> 5] = best;
     }
+}
+
+__device__ __forceinline__ void warp_merge_lists(const unsigned long long* rec, int stride, int P, int k,
+                                                 unsigned long long (&mine)[2]) {
+    if (P <= 32) warp_merge_lists_n<1>(rec, stride, P, k, mine);
+    else if (P <= 64) warp_merge_lists_n<2>(rec, stride, P, k, mine);
+    else if (P <= 160) warp_merge_lists_n<5>(rec, stride, P, k, mine);
+    else warp_merge_lists_n<kMergeSlots>(rec, stride, P, k, mine);
 }
 
 __device__ __forceinline__ float2 warp_merge_ms(const unsigned long long* rec, int stride, int P, int k) {
@@ -226,13 +240,20 @@ __device__ __forceinline__ float2 warp_merge_ms(const unsigned long long* rec, i
 }
 
 // Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
+// The winners are first collected in registers, then written by k lanes at once, so the d2t gathers
+// are one round trip instead of k.
 __device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride) {
     const int lane = threadIdx.x & 31;
     const int k = o.k;
     const float2 ms = warp_merge_ms(rec, stride, P, k);
     const float lse = ms.x + logf(ms.y);
-    warp_merge_lists(rec, stride, P, k, [&](int j, unsigned long long best) {
-        if (lane == 0) {
+    unsigned long long mine[2];
+    warp_merge_lists(rec, stride, P, k, mine);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int j = lane + 32 * e;
+        if (j < k) {
+            const unsigned long long best = mine[e];
             const size_t out = (size_t)m * k + j;
             if (best != 0ull) {
                 const int idx = key_index(best);
@@ -245,7 +266,7 @@ __device__ inline void merge_row_final(const HeadOut& o, int P, int m, const uns
                 if (o.draft_ids) o.draft_ids[out] = -1;
             }
         }
-    });
+    }
     if (lane == 0 && o.lse) o.lse[m] = lse;
 }
 

@@ -217,9 +217,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         const int stride = MP * KS;
         const float2 ms = warp_merge_ms(rec0, stride, P1, k);
         unsigned long long* dst = p.out.recs + ((size_t)cta * M + p.m_begin + m) * KS;
-        warp_merge_lists(rec0, stride, P1, k, [&](int j, unsigned long long best) {
-            if (lane == 0) dst[j] = best;
-        });
+        unsigned long long mine[2];
+        warp_merge_lists(rec0, stride, P1, k, mine);
+        if (lane < k) dst[lane] = mine[0];
+        if (lane + 32 < k) dst[lane + 32] = mine[1];
         if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
     }
 

@@ -8,6 +8,7 @@
 // consecutive vocabulary logits, so the running (max, sum-exp) and the top-k list are thread-private
 // and need no shuffles.  One persistent CTA per SM owns a contiguous range of vocabulary rows:
 //   warp 4   TMA producer: per 64-column k-step one box of h and one box of W into a shared-memory ring
+//   warp 6   fetches h once into shared memory when it fits (else warp 4 streams it per k-step)
 //   warp 5   MMA issuer: four K=16 tcgen05.mma per k-step, tcgen05.commit frees the ring slot;
 //            two accumulator buffers in TMEM so the epilogue of tile t overlaps the MMAs of tile t+1
 //   warps 0-3 epilogue: warp q reads TMEM lanes 32q..32q+31 (draft rows), never stores a logit
@@ -20,9 +21,10 @@
 
 namespace vt {
 
-constexpr int kMmaThreads = 512;               // warps 0-3 epilogue, 4 TMA, 5 MMA; the rest only join the final merge
+constexpr int kMmaThreads = 384;               // warps 0-3 epilogue, 4 TMA, 5 MMA; the rest only join the final merge
 constexpr int kBoxK = 64;                    // bf16 elements per k-step = one 128-byte swizzle row
 constexpr int kMaxStages = 32;
+constexpr size_t kResidentHMax = 96 * 1024;   // h stays in shared memory when its A blocks fit in this
 constexpr int kAccStride = 256;              // TMEM columns between the two accumulator buffers
 
 struct MmaParams {
@@ -35,7 +37,11 @@ struct MmaParams {
     uint32_t stage_bytes;     // A slot + B slot, multiple of 1024
     uint32_t a_slot;          // bytes of the A slot: the pass's rows rounded up to whole 8-row groups
     uint32_t a_tx, b_tx;      // bytes each TMA box delivers
+    int h_resident;           // 1: all of h sits in shared memory for the whole kernel (h_off), one A block per k-step
+    uint32_t h_off;
     uint32_t idesc;
+    int batch_cols;           // vocabulary columns per top-k selection batch (multiple of 32, <= 256)
+    uint32_t tile_floats;     // floats of one warp's transpose buffer
     uint32_t list_off, bar_off, total_smem;   // offsets from the 1024-aligned base
 };
 
@@ -84,6 +90,68 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 }
 
 // ------------------------------------------------------------------------------------------ kernel
+constexpr int kHelpers = 8;                   // warps 1-3 and 7-11 share the top-k selection when one warp owns all draft rows
+constexpr int kMaxBatchCols = 256;            // vocabulary columns the top-k selection takes at a time
+
+// Top-k update of one draft row by a whole warp.  `vals` is the row's logits for `ncols` consecutive
+// vocabulary columns (first column = vocabulary row `col0`), in shared memory; `list` is the row's k best
+// so far (descending keys, 0 = empty) and `tau` the logit of its k-th best (-inf while the list is not
+// full).  Lane L looks at columns L, L+32, ...
+//   1. bound: the 32 lanes form 8 groups of 4; the smallest of the 8 group maxima has at least 8 logits at
+//      or above it, so with k <= 8 nothing below it can be among the k best of these columns;
+//   2. the logits above tau (strictly: a later row loses a tie) and not below the bound are the candidates;
+//      a ballot per column group gives each its slot in `cbuf`, and the current list follows them;
+//   3. every entry of cbuf counts the entries larger than itself - its rank - and the entries of rank < k
+//      form the new list.  Keys are distinct, so ranks are too.  No step depends on the previous candidate,
+//      unlike an insertion loop.
+// Returns the new tau.  All lanes must call it; `cbuf` holds kMaxBatchCols + k keys.
+__device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, int col0, unsigned long long* list,
+                                                  int k, float tau, unsigned long long* cbuf, int lane) {
+    constexpr int NI = kMaxBatchCols / 32;
+    float v[NI];
+    float lmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int c = lane + 32 * i;
+        v[i] = c < ncols ? vals[c] : -INFINITY;
+        lmax = fmaxf(lmax, v[i]);
+    }
+    if (!__any_sync(0xFFFFFFFFu, lmax > tau)) return tau;
+    float bound = -INFINITY;
+    if (k <= 8) {
+        float g = fmaxf(lmax, __shfl_xor_sync(0xFFFFFFFFu, lmax, 1));
+        g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+        g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+        g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 8));
+        bound = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 16));
+    }
+    int n = 0;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const bool is_cand = v[i] > tau && v[i] >= bound;
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, is_cand);
+        if (is_cand) cbuf[n + __popc(m & ((1u << lane) - 1u))] = make_key(v[i], col0 + lane + 32 * i);
+        n += __popc(m);
+    }
+    for (int j = lane; j < k; j += 32) cbuf[n + j] = list[j];      // empty slots are 0 and rank last
+    __syncwarp();
+    const int total = n + k;
+    for (int e = lane; e < total; e += 32) {
+        const unsigned long long key = cbuf[e];
+        int rank = 0;
+        for (int f = 0; f < total; ++f) rank += cbuf[f] > key ? 1 : 0;
+        if (key != 0ull && rank < k) list[rank] = key;
+    }
+    __syncwarp();
+    const unsigned long long kth = list[k - 1];
+    __syncwarp();
+    return kth != 0ull ? key_logit(kth) : -INFINITY;
+}
+
+// Epilogue in two layouts.  tcgen05.ld gives lane = draft row, registers = 32 consecutive vocabulary
+// logits: the running (max, sum-exp) is kept there, thread-private.  For the top-k the logits are turned
+// through shared memory so that a whole warp works on one draft row at a time (warp_topk_update), which
+// keeps all 32 lanes busy when there are only a few draft rows.
 __global__ void __launch_bounds__(kMmaThreads, 1)
 head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
     extern __shared__ unsigned char smem_raw[];
@@ -99,12 +167,13 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
     const int nrows = row_end - row_begin;
     const int ntiles = (nrows + NT - 1) / NT;
 
-    unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [k][128]
+    unsigned long long* epi = reinterpret_cast<unsigned long long*>(smem + p.list_off);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
     const uint32_t bar_full = base + p.bar_off, bar_empty = bar_full + 8u * S;
     const uint32_t bar_accf = bar_empty + 8u * S, bar_acce = bar_accf + 16u, bar_drain = bar_acce + 16u;
-    const uint32_t bar_merge = bar_drain + 8u;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    const uint32_t bar_merge = bar_drain + 8u, bar_h = bar_merge + 8u;
+    const uint32_t bar_sel_ready = bar_h + 8u, bar_sel_done = bar_sel_ready + 8u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 9);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_flag = const_cast<int*>(abort_flag) + 1;
 
@@ -120,11 +189,21 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         }
         mbar_init(bar_drain, 1);
         mbar_init(bar_merge, 1);
+        mbar_init(bar_h, 1);
+        mbar_init(bar_sel_ready, 1);
+        mbar_init(bar_sel_done, kHelpers);
         *abort_flag = 0;
         fence_mbar_init();
     }
-    for (int i = tid; i < k * 128; i += blockDim.x) lists[i] = 0ull;
-    // The MMA always reads 128 A rows; rows past the pass's last row hold whatever follows the A slot in
+    // epilogue scratch: lists [warps * 32][k] keys | candidate staging per warp | transpose buffer per warp
+    for (int i = tid; i < n_epi_warps * 32 * k; i += blockDim.x) epi[i] = 0ull;
+    const bool team_mode = n_epi_warps == 1;       // all draft rows in warp 0: idle warps help with the selection
+    const int n_cbuf = team_mode ? 1 + kHelpers : n_epi_warps;
+    unsigned long long* cands = epi + (size_t)n_epi_warps * 32 * k;
+    float* thr_s = reinterpret_cast<float*>(cands + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K));   // [warps * 32]
+    float* tiles = thr_s + n_epi_warps * 32;
+    for (int i = tid; i < n_epi_warps * 32; i += blockDim.x) thr_s[i] = -INFINITY;
+    // The MMA always reads 128 A rows; rows past the pass's last row hold whatever follows the A block in
     // shared memory.  They only feed TMEM lanes that no thread reads, so they are left as they are.
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -141,50 +220,74 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         atomicOr(&p.out.hdr->status, kStatusTimeout);
     };
 
-    if (warp == 4) {
+    if (warp == 6) {
+        // ------------------------------------------------------------------ resident h: fetched once
+        // Every CTA needs all of h.  One fetch per CTA spreads the 148 CTAs' requests for its lines over
+        // the L2 slices and keeps h out of the per-k-step path.
+        if (lane == 0 && p.h_resident && ntiles > 0) {
+            mbar_arrive_expect_tx(bar_h, p.a_tx * (uint32_t)nk);
+            for (int ks = 0; ks < nk; ++ks)
+                tma_load_2d(base + p.h_off + (uint32_t)ks * p.a_slot, &tmH, ks * kBoxK, p.m_begin, bar_h);
+        }
+    } else if (warp == 4) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            int it = 0, issued = 0;
+            int s = 0, issued = 0;
+            uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * NT;
-                for (int ks = 0; ks < nk; ++ks, ++it) {
-                    const int s = it % S, n = it / S;
-                    if (n > 0 && !mbar_wait(bar_empty + 8u * s, (uint32_t)(n - 1) & 1u)) { fail(); ok = false; break; }
+                for (int ks = 0; ks < nk; ++ks) {
+                    if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
-                    const uint32_t a_dst = base + (uint32_t)s * p.stage_bytes;
-                    mbar_arrive_expect_tx(bar_full + 8u * s, p.a_tx + p.b_tx);
-                    tma_load_2d(a_dst, &tmH, ks * kBoxK, p.m_begin, bar_full + 8u * s);
-                    tma_load_2d(a_dst + p.a_slot, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
-                    issued = it + 1;
+                    const uint32_t dst = base + (uint32_t)s * p.stage_bytes;
+                    if (p.h_resident) {
+                        mbar_arrive_expect_tx(bar_full + 8u * s, p.b_tx);
+                        tma_load_2d(dst, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
+                    } else {
+                        mbar_arrive_expect_tx(bar_full + 8u * s, p.a_tx + p.b_tx);
+                        tma_load_2d(dst, &tmH, ks * kBoxK, p.m_begin, bar_full + 8u * s);
+                        tma_load_2d(dst + p.a_slot, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
+                    }
+                    ++issued;
+                    if (++s == S) { s = 0; ++wrap; }
                 }
             }
             if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
                 for (int i = max(0, issued - S); i < issued; ++i)
                     (void)mbar_wait(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u);
+                if (p.h_resident && ntiles > 0) (void)mbar_wait(bar_h, 0u);
             }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            int it = 0;
+            int s = 0;
+            uint32_t phase = 0;
             bool ok = true;
+            if (p.h_resident && ntiles > 0 && !mbar_wait(bar_h, 0u)) { fail(); ok = false; }
+            const uint64_t desc0 = smem_desc_sw128(base);                      // descriptor of the ring's first byte
+            const uint64_t h_desc0 = smem_desc_sw128(base + p.h_off);
+            const uint32_t stage_units = p.stage_bytes >> 4, a_units = p.a_slot >> 4;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
-                for (int ks = 0; ks < nk; ++ks, ++it) {
-                    const int s = it % S;
-                    if (!mbar_wait(bar_full + 8u * s, (uint32_t)(it / S) & 1u)) { fail(); ok = false; break; }
+                for (int ks = 0; ks < nk; ++ks) {
+                    if (!mbar_wait(bar_full + 8u * s, phase)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = base + (uint32_t)s * p.stage_bytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + p.a_slot);
-#pragma unroll
-                    for (int kk = 0; kk < kBoxK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-                        tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, p.idesc, (ks | kk) != 0);
+                    const uint64_t st_desc = desc0 + (uint64_t)((uint32_t)s * stage_units);
+                    const uint64_t a_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)ks * a_units) : st_desc;
+                    const uint64_t b_desc = p.h_resident ? st_desc : st_desc + a_units;
+                    // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
+                    tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, ks != 0);
+                    tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
+                    tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
+                    tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
                     tc_commit(bar_empty + 8u * s);
+                    if (++s == S) { s = 0; phase ^= 1u; }
                 }
                 if (ok) tc_commit(bar_accf + 8u * buf);
             }
@@ -194,12 +297,17 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             }
         }
     } else if (warp < n_epi_warps) {
-        // ------------------------------------------------------------------ epilogue: lane = draft row
+        // ------------------------------------------------------------------ epilogue: TMEM reader
         const int m_local = warp * 32 + lane;
         const bool live = m_local < p.m_count;
-        float mx = -INFINITY, ssum = 0.0f, thr_x = -INFINITY;
-        unsigned long long* my_list = lists + tid;       // list[j * 128 + tid]
-        int filled = 0;
+        const int rows_here = min(32, p.m_count - warp * 32);          // live draft rows of this warp
+        const int EB = p.batch_cols, EBP = EB + 1;                     // odd row pitch: conflict-free both ways
+        float mx = -INFINITY, ssum = 0.0f;                             // lane = draft row
+        float* tbuf = tiles + (size_t)warp * p.tile_floats;            // tbuf[row * EBP + column in batch]
+        unsigned long long* cbuf = cands + (size_t)warp * (kMaxBatchCols + VT_MAX_K);
+        unsigned long long* lists = epi + (size_t)warp * 32 * k;       // lists[row * k + j]
+        uint32_t batch_no = 0;
+
         for (int t = 0; t < ntiles; ++t) {
             const int buf = t & 1;
             if (!mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u)) { fail(); break; }
@@ -212,48 +320,94 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 uint32_t r[32];
                 tc_ld32(taddr + (uint32_t)c0, r);
                 tc_wait_ld();
-                if (live) {
-                    const int nv = min(32, ncols - c0);
-                    float cmax = -INFINITY;
+                const int nv = min(32, ncols - c0);
+                const int cb = c0 % EB;                                // column of this chunk inside the batch
+                // lane = draft row: log-sum-exp over the chunk; the chunk goes to the transpose buffer
+                float x[32];
+                float cmax = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (c < nv) cmax = fmaxf(cmax, __uint_as_float(r[c]));
+                for (int c = 0; c < 32; ++c) {
+                    x[c] = c < nv ? __uint_as_float(r[c]) : -INFINITY;   // columns past the CTA's rows are not its logits
+                    cmax = fmaxf(cmax, x[c]);
+                    if (lane < rows_here) tbuf[lane * EBP + cb + c] = x[c];
+                }
+                if (live) {
                     if (cmax > mx) {
                         ssum *= __expf(mx - cmax);
                         mx = cmax;
                     }
                     float add = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (c < nv) add += __expf(__uint_as_float(r[c]) - mx);
+                    for (int c = 0; c < 32; ++c) add += __expf(x[c] - mx);
                     ssum += add;
-                    if (cmax > thr_x || filled < k) {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const float x = __uint_as_float(r[c]);
-                            if (c < nv && (x > thr_x || filled < k)) {
-                                const unsigned long long kth = list_insert(my_list, 128, k, make_key(x, row0 + c0 + c));
-                                if (filled < k) ++filled;
-                                if (filled == k) thr_x = key_logit(kth);
-                            }
-                        }
-                    }
                     if (p.out.logits) {
                         float* dst = p.out.logits + (size_t)(p.m_begin + m_local) * Vt + row0 + c0;
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c < nv) dst[c] = __uint_as_float(r[c]);
+                            if (c < nv) dst[c] = x[c];
                     }
                 }
+                // a full batch (or the tile's last chunk): one warp per draft row takes it from here
+                if (cb + 32 >= EB || c0 + 32 >= ncols) {
+                    if (c0 + 32 >= ncols) {          // TMEM is read out: the MMAs of the tile after next may start
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+                    }
+                    __syncwarp();
+                    if (team_mode && lane == 0) mbar_arrive(bar_sel_ready);
+                    const int bvalid = min(min(cb + 32, EB), ncols - (c0 - cb));   // valid columns of the batch
+                    const int bcol0 = row0 + c0 - cb;                              // vocabulary row of its first column
+                    const int team = team_mode ? 1 + kHelpers : 1;
+                    for (int row = 0; row < rows_here; row += team) {
+                        const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
+                                                          thr_s[warp * 32 + row], cbuf, lane);
+                        if (lane == 0) thr_s[warp * 32 + row] = t2;
+                    }
+                    __syncwarp();
+                    if (team_mode && !mbar_wait(bar_sel_done, batch_no & 1u)) { fail(); break; }
+                    ++batch_no;
+                }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
         }
-        if (live) {
-            unsigned long long* rec = p.out.recs + ((size_t)cta * M + p.m_begin + m_local) * ws_slots(k);
-            for (int j = 0; j < k; ++j) rec[j] = my_list[j * 128];
-            rec[k] = pack_ms(mx, ssum);
+        // records: the row's list is contiguous in shared memory, so k lanes copy it out together
+        for (int row = 0; row < rows_here; ++row) {
+            unsigned long long* rec = p.out.recs + ((size_t)cta * M + p.m_begin + warp * 32 + row) * ws_slots(k);
+            for (int j = lane; j < k; j += 32) rec[j] = lists[(size_t)row * k + j];
+        }
+        if (live) p.out.recs[((size_t)cta * M + p.m_begin + m_local) * ws_slots(k) + k] = pack_ms(mx, ssum);
+    } else if (team_mode && warp != 6) {
+        // ------------------------------------------------------------------ selection helpers (warps 1-3, 7-11)
+        // They replay the reader's batch sequence (it depends only on the tile geometry) and take every
+        // (1 + kHelpers)-th draft row of each batch.
+        const int member = warp < 4 ? warp : warp - 3;                 // 1..kHelpers
+        const int rows_here = p.m_count;
+        const int EB = p.batch_cols, EBP = EB + 1;
+        const float* tbuf = tiles;
+        unsigned long long* cbuf = cands + (size_t)member * (kMaxBatchCols + VT_MAX_K);
+        unsigned long long* lists = epi;
+        uint32_t batch_no = 0;
+        bool ok = true;
+        for (int t = 0; t < ntiles && ok; ++t) {
+            const int row0 = row_begin + t * NT;
+            const int ncols = min(NT, row_end - row0);
+            for (int c0 = 0; c0 < ncols; c0 += 32) {
+                const int cb = c0 % EB;
+                if (cb + 32 >= EB || c0 + 32 >= ncols) {
+                    if (!mbar_wait(bar_sel_ready, batch_no & 1u)) { fail(); ok = false; break; }
+                    if (*abort_flag) { ok = false; break; }
+                    const int bvalid = min(min(cb + 32, EB), ncols - (c0 - cb));
+                    const int bcol0 = row0 + c0 - cb;
+                    for (int row = member; row < rows_here; row += 1 + kHelpers) {
+                        const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
+                                                          thr_s[row], cbuf, lane);
+                        if (lane == 0) thr_s[row] = t2;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sel_done);
+                    ++batch_no;
+                }
+            }
         }
     }
 
@@ -265,8 +419,8 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     if (!p.out.fused_merge) return;
     if (publish_and_check_last(p.out.hdr, last_flag)) {
-        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.list_off, bar_merge);   // the ring is free now
-        if (tid == 0) p.out.hdr->ticket = 0u;                                       // ready for the next call
+        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.h_off, bar_merge);   // the ring is free now
+        if (tid == 0) p.out.hdr->ticket = 0u;                                    // ready for the next call
     }
 }
 
@@ -357,25 +511,38 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.a_tx = (uint32_t)mc * 128u;
         p.b_tx = (uint32_t)NT * 128u;
         p.a_slot = (((uint32_t)mc * 128u) + 1023u) & ~1023u;
-        p.stage_bytes = p.a_slot + (((uint32_t)NT * 128u + 1023u) & ~1023u);
+        const uint32_t b_slot = ((uint32_t)NT * 128u + 1023u) & ~1023u;
+        const size_t h_bytes = (size_t)p.nk * p.a_slot;
+        p.h_resident = h_bytes <= kResidentHMax;
+        p.stage_bytes = p.h_resident ? b_slot : p.a_slot + b_slot;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const size_t list_bytes = (size_t)c.out.k * 128 * 8;
-        const size_t bar_bytes = (size_t)(2 * kMaxStages + 6) * 8 + 16;  // sized for the largest stage count
+        // epilogue scratch: lists, candidate staging and a transpose buffer per epilogue warp; the fewer draft
+        // rows a warp has, the more columns it can afford to select from at a time
+        const int epi_warps = (mc + 31) / 32;
+        const int rows_w = std::min(mc, 32);
+        int batch = ((NT + 31) / 32) * 32;
+        while (batch > 32 && (size_t)rows_w * (batch + 1) * 4 > 17 * 1024) batch -= 32;
+        p.batch_cols = batch;
+        p.tile_floats = (uint32_t)(rows_w * (batch + 1));
+        const int n_cbuf = epi_warps == 1 ? 1 + kHelpers : epi_warps;
+        const size_t list_bytes = (((size_t)epi_warps * 32 * c.out.k * 8 + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K) * 8 +
+                                    (size_t)epi_warps * 32 * 4 + (size_t)epi_warps * p.tile_floats * 4) + 127) & ~(size_t)127;
+        const size_t bar_bytes = (size_t)(2 * kMaxStages + 9) * 8 + 16;  // sized for the largest stage count
         const size_t merge_bytes = (size_t)grid * (ws_slots(c.out.k) * 8 + 16);
-        // the MMA reads 128 A rows from the slot's start: keep 16 KB readable past the last stage's A slot
-        const size_t avail = (size_t)kMaxDynSmem - 1024 - list_bytes - bar_bytes - 256 - 16384;
-        int S = (int)std::min<size_t>(kMaxStages, avail / p.stage_bytes);
-        if (S < 2) return VT_ERR_UNSUPPORTED;
+        // Layout from the 1024-aligned base: ring | resident h | 16 KB the MMA may read past the last A block
+        // (it always reads 128 A rows) | lists | barriers.  The pad is never written.
+        const size_t fixed = 1024 + (p.h_resident ? h_bytes : 0) + 16384 + list_bytes + bar_bytes + 256;
+        if (fixed + 2 * (size_t)p.stage_bytes > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
+        int S = (int)std::min<size_t>(kMaxStages, ((size_t)kMaxDynSmem - fixed) / p.stage_bytes);
         size_t ring = (size_t)S * p.stage_bytes;
-        if (ring < 16384 + (size_t)p.stage_bytes) ring = 16384 + p.stage_bytes;
         if (ring < merge_bytes) ring = (merge_bytes + 1023) & ~(size_t)1023;
-        if (ring + list_bytes + bar_bytes + 1024 + 256 > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
+        if (ring + fixed > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
         p.n_stages = S;
-        p.list_off = (uint32_t)ring;
-        p.bar_off = (uint32_t)((ring + list_bytes + 127) & ~(size_t)127);
-        const size_t a_overread = (size_t)(S - 1) * p.stage_bytes + 16384;     // last A slot + 128 rows
-        p.total_smem = (uint32_t)(std::max<size_t>(p.bar_off + bar_bytes, a_overread) + 1024);
+        p.h_off = (uint32_t)ring;
+        p.list_off = (uint32_t)(ring + (p.h_resident ? h_bytes : 0) + 16384);
+        p.bar_off = (uint32_t)((p.list_off + list_bytes + 127) & ~(size_t)127);
+        p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
 
         head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmH, p);
         count_launch();
