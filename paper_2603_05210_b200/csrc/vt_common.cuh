@@ -90,7 +90,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Waits for the phase with the given parity to complete, for at most kWaitLimitNs.
 // Returns false when the limit ran out (the caller records it and unwinds; nothing spins forever).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < 64; ++i)                       // the common case: no clock read on the way
+        if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {

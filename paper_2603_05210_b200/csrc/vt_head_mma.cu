@@ -32,7 +32,9 @@ struct MmaParams {
     int m_begin, m_count;     // draft rows of this pass
     int d;
     int NT;                   // vocabulary rows per tile (multiple of 16, <= 256)
-    int nk;                   // k-steps per tile
+    int nk;                   // 64-column k-blocks per tile
+    int kb_per_stage;         // k-blocks one ring stage holds (one barrier hand-over per stage)
+    uint32_t blk_bytes;       // bytes of one k-block in a stage: (A slot +) B slot, multiple of 1024
     int n_stages;
     uint32_t stage_bytes;     // A slot + B slot, multiple of 1024
     uint32_t a_slot;          // bytes of the A slot: the pass's rows rounded up to whole 8-row groups
@@ -104,9 +106,10 @@ constexpr int kMaxBatchCols = 256;            // vocabulary columns the top-k se
 //   3. every entry of cbuf counts the entries larger than itself - its rank - and the entries of rank < k
 //      form the new list.  Keys are distinct, so ranks are too.  No step depends on the previous candidate,
 //      unlike an insertion loop.
+// The same pass folds the columns into the row's running (max, sum-exp) in *ms.
 // Returns the new tau.  All lanes must call it; `cbuf` holds kMaxBatchCols + k keys.
 __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, int col0, unsigned long long* list,
-                                                  int k, float tau, unsigned long long* cbuf, int lane) {
+                                                  int k, float tau, unsigned long long* cbuf, float2* ms, int lane) {
     constexpr int NI = kMaxBatchCols / 32;
     float v[NI];
     float lmax = -INFINITY;
@@ -115,6 +118,17 @@ __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, 
         const int c = lane + 32 * i;
         v[i] = c < ncols ? vals[c] : -INFINITY;
         lmax = fmaxf(lmax, v[i]);
+    }
+    {   // running log-sum-exp of the row: (max, sum of exp(x - max)), folded over these columns by the warp
+        const float2 old = *ms;
+        const float bmax = warp_max_f32(lmax);
+        const float nmx = fmaxf(old.x, bmax);
+        float add = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NI; ++i) add += __expf(v[i] - nmx);      // exp(-inf) = 0 for the padding
+        add = warp_sum_f32(add);
+        __syncwarp();
+        if (lane == 0) *ms = make_float2(nmx, old.y * __expf(old.x - nmx) + add);
     }
     if (!__any_sync(0xFFFFFFFFu, lmax > tau)) return tau;
     float bound = -INFINITY;
@@ -201,8 +215,12 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
     const int n_cbuf = team_mode ? 1 + kHelpers : n_epi_warps;
     unsigned long long* cands = epi + (size_t)n_epi_warps * 32 * k;
     float* thr_s = reinterpret_cast<float*>(cands + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K));   // [warps * 32]
-    float* tiles = thr_s + n_epi_warps * 32;
-    for (int i = tid; i < n_epi_warps * 32; i += blockDim.x) thr_s[i] = -INFINITY;
+    float2* ms_s = reinterpret_cast<float2*>(thr_s + n_epi_warps * 32);                               // [warps * 32]
+    float* tiles = reinterpret_cast<float*>(ms_s + n_epi_warps * 32);
+    for (int i = tid; i < n_epi_warps * 32; i += blockDim.x) {
+        thr_s[i] = -INFINITY;
+        ms_s[i] = make_float2(-INFINITY, 0.0f);
+    }
     // The MMA always reads 128 A rows; rows past the pass's last row hold whatever follows the A block in
     // shared memory.  They only feed TMEM lanes that no thread reads, so they are left as they are.
     if (warp == 5) {
@@ -237,17 +255,20 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * NT;
-                for (int ks = 0; ks < nk; ++ks) {
+                for (int ks = 0; ks < nk; ks += p.kb_per_stage) {
                     if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
-                    const uint32_t dst = base + (uint32_t)s * p.stage_bytes;
-                    if (p.h_resident) {
-                        mbar_arrive_expect_tx(bar_full + 8u * s, p.b_tx);
-                        tma_load_2d(dst, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
-                    } else {
-                        mbar_arrive_expect_tx(bar_full + 8u * s, p.a_tx + p.b_tx);
-                        tma_load_2d(dst, &tmH, ks * kBoxK, p.m_begin, bar_full + 8u * s);
-                        tma_load_2d(dst + p.a_slot, &tmW, ks * kBoxK, row0, bar_full + 8u * s);
+                    const int nb = min(p.kb_per_stage, nk - ks);
+                    const uint32_t bar = bar_full + 8u * s;
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (p.h_resident ? p.b_tx : p.a_tx + p.b_tx));
+                    for (int kb = 0; kb < nb; ++kb) {
+                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
+                        if (p.h_resident) {
+                            tma_load_2d(dst, &tmW, (ks + kb) * kBoxK, row0, bar);
+                        } else {
+                            tma_load_2d(dst, &tmH, (ks + kb) * kBoxK, p.m_begin, bar);
+                            tma_load_2d(dst + p.a_slot, &tmW, (ks + kb) * kBoxK, row0, bar);
+                        }
                     }
                     ++issued;
                     if (++s == S) { s = 0; ++wrap; }
@@ -268,24 +289,27 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             if (p.h_resident && ntiles > 0 && !mbar_wait(bar_h, 0u)) { fail(); ok = false; }
             const uint64_t desc0 = smem_desc_sw128(base);                      // descriptor of the ring's first byte
             const uint64_t h_desc0 = smem_desc_sw128(base + p.h_off);
-            const uint32_t stage_units = p.stage_bytes >> 4, a_units = p.a_slot >> 4;
+            const uint32_t stage_units = p.stage_bytes >> 4, a_units = p.a_slot >> 4, blk_units = p.blk_bytes >> 4;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
-                for (int ks = 0; ks < nk; ++ks) {
+                for (int ks = 0; ks < nk; ks += p.kb_per_stage) {
                     if (!mbar_wait(bar_full + 8u * s, phase)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t st_desc = desc0 + (uint64_t)((uint32_t)s * stage_units);
-                    const uint64_t a_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)ks * a_units) : st_desc;
-                    const uint64_t b_desc = p.h_resident ? st_desc : st_desc + a_units;
-                    // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
-                    tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, ks != 0);
-                    tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
-                    tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
-                    tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                    const int nb = min(p.kb_per_stage, nk - ks);
+                    for (int kb = 0; kb < nb; ++kb) {
+                        const uint64_t blk_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * blk_units);
+                        const uint64_t a_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)(ks + kb) * a_units) : blk_desc;
+                        const uint64_t b_desc = p.h_resident ? blk_desc : blk_desc + a_units;
+                        // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
+                        tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                    }
                     tc_commit(bar_empty + 8u * s);
                     if (++s == S) { s = 0; phase ^= 1u; }
                 }
@@ -302,7 +326,6 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         const bool live = m_local < p.m_count;
         const int rows_here = min(32, p.m_count - warp * 32);          // live draft rows of this warp
         const int EB = p.batch_cols, EBP = EB + 1;                     // odd row pitch: conflict-free both ways
-        float mx = -INFINITY, ssum = 0.0f;                             // lane = draft row
         float* tbuf = tiles + (size_t)warp * p.tile_floats;            // tbuf[row * EBP + column in batch]
         unsigned long long* cbuf = cands + (size_t)warp * (kMaxBatchCols + VT_MAX_K);
         unsigned long long* lists = epi + (size_t)warp * 32 * k;       // lists[row * k + j]
@@ -322,29 +345,15 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 tc_wait_ld();
                 const int nv = min(32, ncols - c0);
                 const int cb = c0 % EB;                                // column of this chunk inside the batch
-                // lane = draft row: log-sum-exp over the chunk; the chunk goes to the transpose buffer
-                float x[32];
-                float cmax = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    x[c] = c < nv ? __uint_as_float(r[c]) : -INFINITY;   // columns past the CTA's rows are not its logits
-                    cmax = fmaxf(cmax, x[c]);
-                    if (lane < rows_here) tbuf[lane * EBP + cb + c] = x[c];
-                }
+                // lane = draft row: the chunk goes to the transpose buffer (columns past the CTA's rows are not its logits)
                 if (live) {
-                    if (cmax > mx) {
-                        ssum *= __expf(mx - cmax);
-                        mx = cmax;
-                    }
-                    float add = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) add += __expf(x[c] - mx);
-                    ssum += add;
+                    for (int c = 0; c < 32; ++c) tbuf[lane * EBP + cb + c] = c < nv ? __uint_as_float(r[c]) : -INFINITY;
                     if (p.out.logits) {
                         float* dst = p.out.logits + (size_t)(p.m_begin + m_local) * Vt + row0 + c0;
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c < nv) dst[c] = x[c];
+                            if (c < nv) dst[c] = __uint_as_float(r[c]);
                     }
                 }
                 // a full batch (or the tile's last chunk): one warp per draft row takes it from here
@@ -361,7 +370,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                     const int team = team_mode ? 1 + kHelpers : 1;
                     for (int row = 0; row < rows_here; row += team) {
                         const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
-                                                          thr_s[warp * 32 + row], cbuf, lane);
+                                                          thr_s[warp * 32 + row], cbuf, ms_s + warp * 32 + row, lane);
                         if (lane == 0) thr_s[warp * 32 + row] = t2;
                     }
                     __syncwarp();
@@ -375,7 +384,10 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             unsigned long long* rec = p.out.recs + ((size_t)cta * M + p.m_begin + warp * 32 + row) * ws_slots(k);
             for (int j = lane; j < k; j += 32) rec[j] = lists[(size_t)row * k + j];
         }
-        if (live) p.out.recs[((size_t)cta * M + p.m_begin + m_local) * ws_slots(k) + k] = pack_ms(mx, ssum);
+        if (live) {
+            const float2 ms = ms_s[warp * 32 + lane];
+            p.out.recs[((size_t)cta * M + p.m_begin + m_local) * ws_slots(k) + k] = pack_ms(ms.x, ms.y);
+        }
     } else if (team_mode && warp != 6) {
         // ------------------------------------------------------------------ selection helpers (warps 1-3, 7-11)
         // They replay the reader's batch sequence (it depends only on the tile geometry) and take every
@@ -400,7 +412,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                     const int bcol0 = row0 + c0 - cb;
                     for (int row = member; row < rows_here; row += 1 + kHelpers) {
                         const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
-                                                          thr_s[row], cbuf, lane);
+                                                          thr_s[row], cbuf, ms_s + row, lane);
                         if (lane == 0) thr_s[row] = t2;
                     }
                     __syncwarp();
@@ -458,8 +470,9 @@ static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, in
     return cr == CUDA_SUCCESS ? VT_OK : driver_fail((int)cr);
 }
 
-// Tile height: a multiple of 16 in [16, 256] that covers ceil(Vt / grid) rows with the least padding,
-// preferring taller tiles (fewer accumulator hand-overs) among equals.
+// Tile height: a multiple of 16 in [16, 256] that covers ceil(Vt / grid) rows with the least padding (rows
+// past the CTA's range that a tile still loads are wasted HBM traffic), preferring taller tiles among
+// equals: fewer accumulator hand-overs and fewer selection batches per draft row.
 static int choose_tile_rows(int rows_per_cta) {
     int best = 16, best_pad = 1 << 30;
     for (int nt = 16; nt <= 256; nt += 16) {
@@ -514,7 +527,11 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         const uint32_t b_slot = ((uint32_t)NT * 128u + 1023u) & ~1023u;
         const size_t h_bytes = (size_t)p.nk * p.a_slot;
         p.h_resident = h_bytes <= kResidentHMax;
-        p.stage_bytes = p.h_resident ? b_slot : p.a_slot + b_slot;
+        p.blk_bytes = p.h_resident ? b_slot : p.a_slot + b_slot;
+        // a stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height
+        p.kb_per_stage = std::max(1, std::min(4, (int)((28 * 1024 + p.blk_bytes / 2) / p.blk_bytes)));
+        p.kb_per_stage = std::min(p.kb_per_stage, p.nk);
+        p.stage_bytes = p.blk_bytes * p.kb_per_stage;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // epilogue scratch: lists, candidate staging and a transpose buffer per epilogue warp; the fewer draft
@@ -527,7 +544,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.tile_floats = (uint32_t)(rows_w * (batch + 1));
         const int n_cbuf = epi_warps == 1 ? 1 + kHelpers : epi_warps;
         const size_t list_bytes = (((size_t)epi_warps * 32 * c.out.k * 8 + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K) * 8 +
-                                    (size_t)epi_warps * 32 * 4 + (size_t)epi_warps * p.tile_floats * 4) + 127) & ~(size_t)127;
+                                    (size_t)epi_warps * 32 * 12 + (size_t)epi_warps * p.tile_floats * 4) + 127) & ~(size_t)127;
         const size_t bar_bytes = (size_t)(2 * kMaxStages + 9) * 8 + 16;  // sized for the largest stage count
         const size_t merge_bytes = (size_t)grid * (ws_slots(c.out.k) * 8 + 16);
         // Layout from the 1024-aligned base: ring | resident h | 16 KB the MMA may read past the last A block
