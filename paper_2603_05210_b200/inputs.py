@@ -39,7 +39,7 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 def _normal_block(args):
     seed, block, n, std = args
-    g = np.random.Generator(np.random.Philox(np.random.SeedSequence([int(seed), int(block)])))
+    g = np.random.Generator(np.random.Philox(np.random.SeedSequence([int(seed), 1, int(block)])))
     x = g.standard_normal(n, dtype=np.float32)
     if std != 1.0:
         x *= np.float32(std)
@@ -50,7 +50,8 @@ def normal_bf16(shape, std: float, seed: int, threads: int | None = None) -> np.
     """bf16 bit patterns of N(0, std^2) samples, drawn in fixed-size blocks.
 
     Each block of ``_BLOCK`` elements has its own Philox stream keyed by
-    ``(seed, block index)``, so the result does not depend on the thread count.
+    ``(seed, 1, block index)``, so the result does not depend on the thread count.  Hidden states
+    use the key ``(seed, 2)`` and token streams ``(seed, 3)``: no two generators share a stream.
     """
     n = int(np.prod(shape))
     out = np.empty(n, dtype=np.uint16)
@@ -68,7 +69,7 @@ def normal_bf16(shape, std: float, seed: int, threads: int | None = None) -> np.
 
 def hidden_states_bf16(M: int, d: int, seed: int, row_scale: tuple[float, float] | None = None) -> np.ndarray:
     """``h`` [M, d]: N(0,1) rows, optionally each multiplied by a U(lo, hi) scale, as bf16 bits."""
-    g = np.random.Generator(np.random.Philox(np.random.SeedSequence([int(seed), 0x68])))
+    g = np.random.Generator(np.random.Philox(np.random.SeedSequence([int(seed), 2])))
     x = g.standard_normal((M, d), dtype=np.float32)
     if row_scale is not None:
         lo, hi = row_scale
@@ -82,7 +83,7 @@ def zipf_token_stream(V: int, s: float, N: int, seed: int) -> np.ndarray:
     ``perm`` is a seeded permutation of the ids, so frequent tokens are scattered
     over the id range the way a tokenizer's frequent ids are.
     """
-    g = np.random.Generator(np.random.PCG64(np.random.SeedSequence([int(seed), 0x7A])))
+    g = np.random.Generator(np.random.PCG64(np.random.SeedSequence([int(seed), 3])))
     perm = g.permutation(V).astype(np.int32)
     w = np.arange(1, V + 1, dtype=np.float64) ** (-float(s))
     cdf = np.cumsum(w)
