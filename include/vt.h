@@ -161,6 +161,30 @@ vt_status vt_coverage(const int32_t* token_ids, int64_t N,
                       uint64_t* covered_out, double* fraction_out,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* vt_coverage for callers that must not allocate device memory.  (The paper has no counterpart: this
+ * entry point exists for integration, not for the method.)
+ *
+ * Who needs it: code that runs inside someone else's serving loop - an engine plugin that is handed a
+ * stream and device pointers but does not own an allocator, or a process whose memory pool has been
+ * reserved up front so that a late cudaMalloc would either fail or stall every stream on the device
+ * while it runs.  vt_coverage asks such a caller for a scratch buffer it cannot provide; this variant
+ * keeps the membership bitmap and the counters in a fixed array inside the library instead, and makes
+ * no cudaMalloc / cudaFree call of its own.
+ *
+ * Same arguments, results and errors as vt_coverage, minus the workspace, with these differences:
+ *  - V_full may be at most 262,144 (the built-in bitmap is 32 KiB; with its counters the array takes
+ *    33,024 bytes on every device that loads the library, until the process ends).  A larger V_full
+ *    returns VT_ERR_SHAPE and launches nothing.
+ *  - The first call on a device looks up the array's device address and remembers it.  Make that first
+ *    call on each device outside any stream capture.
+ *  - All calls on a device share the one array.  Each call clears it before use, so results do not
+ *    depend on earlier calls, but two calls whose GPU work can overlap (different streams, different
+ *    host threads) race on it: keep them ordered.
+ * SYNCHRONISES the stream once to return the count, like vt_coverage. */
+vt_status vt_coverage_static(const int32_t* token_ids, int64_t N,
+                             const int32_t* keep_ids, int V_trim, int V_full,
+                             uint64_t* covered_out, double* fraction_out, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Test and inspection entry points (same kernels as the calls above).
  */

@@ -37,6 +37,7 @@ SYMBOLS = {
     "vt_draft_head_host": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _sz, _p]),
     "vt_last_status": (_i, [_p, _p]),
     "vt_coverage": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p, _sz, _p]),
+    "vt_coverage_static": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p]),
     "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
     "vt_last_launch_count": (_i, []),
@@ -195,6 +196,20 @@ def vt_coverage(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int,
                              keep_ids.data_ptr(), keep_ids.numel(), V_full,
                              ctypes.addressof(covered), ctypes.addressof(frac),
                              workspace.data_ptr(), workspace.numel(), _stream()), "vt_coverage")
+    return int(covered.value), float(frac.value)
+
+
+def vt_coverage_static(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int) -> tuple[int, float]:
+    """``vt_coverage`` without a workspace: the library's built-in scratch is used and nothing is allocated
+    here or in the library (for callers that may not allocate; V_full <= 262,144; calls must not overlap)."""
+    token_ids = _i32(token_ids, "token_ids")
+    keep_ids = _i32(keep_ids, "keep_ids")
+    covered = ctypes.c_uint64(0)
+    frac = ctypes.c_double(0.0)
+    _check(lib().vt_coverage_static(token_ids.data_ptr() if token_ids.numel() else None, token_ids.numel(),
+                                    keep_ids.data_ptr(), keep_ids.numel(), V_full,
+                                    ctypes.addressof(covered), ctypes.addressof(frac), _stream()),
+           "vt_coverage_static")
     return int(covered.value), float(frac.value)
 
 

@@ -186,4 +186,56 @@ vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full,
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
 }
 
+// ------------------------------------------------------------------------------------------
+// Coverage without caller-provided scratch: the bitmap and the counters live in a fixed array that is
+// part of the library image on every device that loads it.
+// ------------------------------------------------------------------------------------------
+constexpr int kStaticCoverageMaxV = 262144;    // largest V_full vt_coverage_static accepts (bitmap: 32 KiB)
+static __device__ __align__(256) unsigned char g_static_coverage[sizeof(CoverageCounters) + kStaticCoverageMaxV / 8];
+
+// Device address of g_static_coverage on the current device.  In host code the array's name is only a
+// handle for the runtime, not a pointer a kernel could use, so the address is asked for once per device
+// (with that device current) and remembered.
+static vt_status static_coverage_address(void** out) {
+    static void* cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_coverage);
+        if (e != cudaSuccess) return cuda_fail(e);
+        cached[dev] = ptr;
+    }
+    *out = cached[dev];
+    return VT_OK;
+}
+
 }  // namespace vt
+
+extern "C" vt_status vt_coverage_static(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim,
+                                        int V_full, uint64_t* covered_out, double* fraction_out, void* stream) {
+    using namespace vt;
+    if (!keep_ids || (!token_ids && N > 0)) return VT_ERR_NULL;
+    if (V_full < 1 || V_trim < 1 || N < 0) return VT_ERR_SHAPE;
+    if (V_full > kStaticCoverageMaxV) return VT_ERR_SHAPE;       // the built-in scratch holds no larger bitmap
+    if (N == 0) return VT_ERR_EMPTY;
+    if ((reinterpret_cast<uintptr_t>(token_ids) & 3) || (reinterpret_cast<uintptr_t>(keep_ids) & 3)) return VT_ERR_ALIGN;
+    void* scratch = nullptr;
+    vt_status r = static_coverage_address(&scratch);
+    if (r != VT_OK) return r;
+    cudaStream_t st = (cudaStream_t)stream;
+    r = launch_keep_bitmap(keep_ids, V_trim, V_full, scratch, st);   // starts by zeroing counters and bitmap
+    if (r != VT_OK) return r;
+    r = launch_coverage_count(token_ids, N, V_full, scratch, st);
+    if (r != VT_OK) return r;
+    CoverageCounters c;
+    cudaError_t e = cudaMemcpyAsync(&c, scratch, sizeof c, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (covered_out) *covered_out = c.covered;
+    if (fraction_out) *fraction_out = (double)c.covered / (double)N;
+    return VT_OK;
+}
