@@ -97,6 +97,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x: float, dist, device) -> float:
+    """The slowest rank's figure: every multi-GPU number is the max over ranks."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_us_per_call(us_per_call_slowest_rank: float, world: int) -> float:
+    """N replicas each finish one call in that time: the job's time per call is 1/N of it (weak scaling)."""
+    return us_per_call_slowest_rank / world
+
+
 def to_dev(a, torch, dtype=None):
     t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
     return t.view(dtype) if dtype is not None else t
@@ -187,13 +202,11 @@ def run_ours(args):
     sampler.start()
     ms, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup)
     clocks = sampler.stop()
+    ms = max_over_ranks(ms, dist, "cuda")
     if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
         dist.barrier()
     us_per_call_rank = ms * 1000.0 / args.steps
-    value = us_per_call_rank / world                  # whole job: N replicas finish N calls in that time
+    value = whole_job_us_per_call(us_per_call_rank, world)
     bytes_call = head_bytes(d, Vt, M, k)
     achieved = bytes_call / (us_per_call_rank * 1e-6) / 1e9
 
@@ -210,10 +223,7 @@ def run_ours(args):
     for i in range(e2e_steps):
         vt.vt_draft_head_host(h_host, copies[i % nc], d2t, k, tid_h, lp_h, hws)
     e2e_us = (time.perf_counter() - t0) * 1e6 / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_us], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_us = float(t.item())
+    e2e_us = max_over_ranks(e2e_us, dist, "cuda")
 
     line = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -47,7 +47,7 @@ typedef enum vt_status {
 /* Which contraction kernel vt_draft_head_path / vt_debug_logits run. */
 typedef enum vt_path {
     VT_PATH_AUTO = 0,      /* chosen from M and d                                                     */
-    VT_PATH_GEMV = 1,      /* CUDA-core streaming GEMV; M <= 8 per pass and d <= 8192                 */
+    VT_PATH_GEMV = 1,      /* CUDA-core streaming GEMV; 4 draft rows per pass, d <= 8192              */
     VT_PATH_MMA = 2        /* tcgen05 tensor-core GEMM with TMEM accumulators; any M                   */
 } vt_path;
 
@@ -64,9 +64,9 @@ int vt_last_cuda_error(void);
  *   W_trim[i, :] = W_full[keep_ids[i], :]      for i in [0, V_trim),  a bit copy of bf16 rows
  *
  *   W_full   dev  [V_full, d] bf16 row-major, 16-byte aligned
- *   keep_ids dev  [V_trim] int32, each in [0, V_full), pairwise distinct (not checked here:
- *                 vt_validate_keep_ids does that; an out-of-range id is skipped and sets
- *                 VT_ERR_RANGE in no status word - validate first)
+ *   keep_ids dev  [V_trim] int32, each in [0, V_full), pairwise distinct.  This call does not check that
+ *                 (vt_validate_keep_ids does, and synchronises to do so); a row whose id is out of range
+ *                 is left unwritten
  *   W_trim   dev  [V_trim, d] bf16 row-major, caller-allocated, 16-byte aligned, must not
  *                 overlap W_full
  * Asynchronous.  VT_ERR_NULL / VT_ERR_SHAPE / VT_ERR_ALIGN / VT_ERR_CUDA.
@@ -191,7 +191,7 @@ vt_status vt_coverage_static(const int32_t* token_ids, int64_t N,
 
 /* The head contraction alone (Section 2.3), with the epilogue storing x[m, i] as fp32:
  * logits dev [M, V_trim] row-major (out).  Runs the same contraction code as vt_draft_head
- * on the chosen path; workspace as for vt_draft_head with k = 1. */
+ * on the chosen path; workspace as for vt_draft_head with k = 2 (vt_workspace_bytes(M, 2)). */
 vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V_trim,
                           float* logits, void* workspace, size_t workspace_bytes,
                           void* stream, int path);
