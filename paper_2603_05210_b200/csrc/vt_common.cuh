@@ -13,10 +13,13 @@ namespace vt {
 // ------------------------------------------------------------------------------------------
 // Workspace of a draft-head call:
 //   [0, 256)                          WsHeader
-//   recs [kMaxParts][M][KS] u64       per-CTA partial results, one record per (CTA, draft row):
+//   recs [kMaxParts][pitch] u64       per-CTA partial results: M records of KS slots, then padding
 //                                     slots 0..k-1  top-k list as sortable keys, descending, 0-padded
 //                                     slot  k       (running max, sum of exp(x - max)) as two floats
-//                                     KS = k + 1 rounded up to even, so every record is 16-byte aligned
+//                                     KS = k + 1 rounded up to even, so every record is 16-byte aligned;
+//                                     pitch = M * KS, plus 2 when that makes pitch / 2 odd: all CTAs' records
+//                                     can then be copied to shared memory as one block and read there by 32
+//                                     lanes (one CTA each) with at most 2-way bank conflicts
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxParts = 256;             // upper bound on CTAs that contribute partials
 constexpr size_t kHeaderBytes = 256;
@@ -31,10 +34,17 @@ static_assert(sizeof(WsHeader) == kHeaderBytes, "header is one 256-byte line");
 constexpr unsigned int kStatusTimeout = 1u;
 
 __host__ __device__ inline int ws_slots(int k) { return (k + 2) & ~1; }
+__host__ __device__ inline int ws_pitch(int M, int k) {
+    const int raw = M * ws_slots(k);
+    return ((raw >> 1) & 1) ? raw : raw + 2;
+}
 __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
-    size_t b = kHeaderBytes + (size_t)kMaxParts * M * ws_slots(k) * 8;
+    size_t b = kHeaderBytes + (size_t)kMaxParts * ws_pitch(M, k) * 8;
     return (b + 255) & ~(size_t)255;
 }
+
+// Record of (CTA p, draft row m).
+#define VT_REC(o, p, m) ((o).recs + (size_t)(p) * ws_pitch((o).M, (o).k) + (size_t)(m) * ws_slots((o).k))
 
 struct HeadOut {
     const int32_t* d2t;   // null: report draft indices as target ids
@@ -229,45 +239,112 @@ __device__ __forceinline__ void warp_merge_lists(const unsigned long long* rec, 
 
 __device__ __forceinline__ float2 warp_merge_ms(const unsigned long long* rec, int stride, int P, int k) {
     const int lane = threadIdx.x & 31;
+    float2 v[kMergeSlots];
     float mx = -INFINITY;
-    for (int p = lane; p < P; p += 32) mx = fmaxf(mx, unpack_ms(rec[(size_t)p * stride + k]).x);
+#pragma unroll
+    for (int q = 0; q < kMergeSlots; ++q) {
+        const int p = lane + 32 * q;
+        v[q] = p < P ? unpack_ms(rec[(size_t)p * stride + k]) : make_float2(-INFINITY, 0.0f);
+        mx = fmaxf(mx, v[q].x);
+    }
     mx = warp_max_f32(mx);
     float s = 0.0f;
-    for (int p = lane; p < P; p += 32) {
-        const float2 v = unpack_ms(rec[(size_t)p * stride + k]);
-        if (v.y > 0.0f) s += v.y * __expf(v.x - mx);
-    }
+#pragma unroll
+    for (int q = 0; q < kMergeSlots; ++q)
+        if (v[q].y > 0.0f) s += v[q].y * __expf(v[q].x - mx);
     return make_float2(mx, warp_sum_f32(s));
 }
 
-// Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
-// The winners are first collected in registers, then written by k lanes at once, so the d2t gathers
-// are one round trip instead of k.
-__device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride) {
+constexpr int kMergeCand = 256;      // candidate slots per warp in warp_select_topk
+
+// The k best keys of P descending lists (rec[p * stride + j], 0 = empty) without k sequential rounds.
+//   1. bound: every lane takes the best head of its lists; the lanes that have one are packed to the
+//      front and fall into G groups (lane % G; G = 8, 16 or 32 >= k); the smallest group maximum has at
+//      least k keys at or above it, so a key whose logit word is below that bound's cannot be among the
+//      k best;
+//   2. the remaining keys (typically one or two dozen) are packed into `cbuf` with ballots, walking the
+//      lists from their heads and stopping at the first depth where no list has a candidate left;
+//   3. each candidate counts the candidates above it: that is its rank, and emit(rank, key) is called
+//      for rank < k by the lane that holds the candidate.
+// Falls back to the round-based merge when the bound does not apply (k > 32, or fewer than G lists) or the
+// candidates do not fit.  emit may be called by several lanes at once, each with a different rank.
+template <class Emit>
+__device__ __forceinline__ void warp_select_topk(const unsigned long long* rec, int stride, int P, int k,
+                                                 unsigned long long* cbuf, Emit emit) {
     const int lane = threadIdx.x & 31;
-    const int k = o.k;
-    const float2 ms = warp_merge_ms(rec, stride, P, k);
-    const float lse = ms.x + logf(ms.y);
-    unsigned long long mine[2];
-    warp_merge_lists(rec, stride, P, k, mine);
+    bool fast = k <= 32;
+    int n = 0;
+    if (fast) {
+        uint32_t lhead = 0;
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-        const int j = lane + 32 * e;
-        if (j < k) {
-            const unsigned long long best = mine[e];
-            const size_t out = (size_t)m * k + j;
-            if (best != 0ull) {
-                const int idx = key_index(best);
-                o.target_ids[out] = o.d2t ? __ldg(&o.d2t[idx]) : idx;
-                o.logprobs[out] = key_logit(best) - lse;
-                if (o.draft_ids) o.draft_ids[out] = idx;
-            } else {   // fewer than k candidates exist only if a wait ran out upstream
-                o.target_ids[out] = -1;
-                o.logprobs[out] = -INFINITY;
-                if (o.draft_ids) o.draft_ids[out] = -1;
+        for (int q = 0; q < kMergeSlots; ++q) {
+            const int p = lane + 32 * q;
+            if (p < P) lhead = max(lhead, (uint32_t)(rec[(size_t)p * stride] >> 32));
+        }
+        // pack the lanes that own a non-empty list to the front, then lane L belongs to group L % G
+        const int G = k <= 8 ? 8 : k <= 16 ? 16 : 32;
+        const unsigned int have = __ballot_sync(0xFFFFFFFFu, lhead != 0u);
+        const int nvalid = __popc(have);
+        const unsigned int src = __fns(have, 0, lane + 1);
+        uint32_t v = __shfl_sync(0xFFFFFFFFu, lhead, src & 31);
+        if (lane >= nvalid) v = 0u;
+        fast = nvalid >= G;                                   // every group has a key: G >= k keys are >= the bound
+        if (G <= 16) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 16));
+        if (G <= 8) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 8));
+        const uint32_t bound = __reduce_min_sync(0xFFFFFFFFu, lane < G ? v : 0xFFFFFFFFu);
+        for (int q = 0; q < kMergeSlots && q * 32 < P && fast; ++q) {
+            const int p = lane + 32 * q;
+            for (int j = 0; j < k; ++j) {
+                const unsigned long long key = p < P ? rec[(size_t)p * stride + j] : 0ull;
+                const bool is_cand = key != 0ull && (uint32_t)(key >> 32) >= bound;
+                const unsigned int m = __ballot_sync(0xFFFFFFFFu, is_cand);
+                if (m == 0u) break;                           // lists descend: nothing deeper qualifies
+                if (n + __popc(m) > kMergeCand) { fast = false; break; }
+                if (is_cand) cbuf[n + __popc(m & ((1u << lane) - 1u))] = key;
+                n += __popc(m);
             }
         }
     }
+    __syncwarp();
+    if (fast) {
+        for (int e = lane; e < n; e += 32) {
+            const unsigned long long key = cbuf[e];
+            int rank = 0;
+#pragma unroll 4
+            for (int f = 0; f < n; ++f) rank += cbuf[f] > key ? 1 : 0;
+            if (rank < k) emit(rank, key);
+        }
+        for (int j = n + lane; j < k; j += 32) emit(j, 0ull);     // fewer than k keys exist at all
+    } else {
+        unsigned long long mine[2];
+        warp_merge_lists(rec, stride, P, k, mine);
+        if (lane < k) emit(lane, mine[0]);
+        if (lane + 32 < k) emit(lane + 32, mine[1]);
+    }
+    __syncwarp();
+}
+
+// Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
+// Winners are written by the lanes that hold them, so the d2t gathers are one round trip, not k.
+__device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride,
+                                       unsigned long long* cbuf) {
+    const int lane = threadIdx.x & 31;
+    const int k = o.k;
+    const float2 ms = warp_merge_ms(rec, stride, P, k);
+    const float lse = ms.x + __logf(ms.y);
+    warp_select_topk(rec, stride, P, k, cbuf, [&](int j, unsigned long long best) {
+        const size_t out = (size_t)m * k + j;
+        if (best != 0ull) {
+            const int idx = key_index(best);
+            o.target_ids[out] = o.d2t ? __ldg(&o.d2t[idx]) : idx;
+            o.logprobs[out] = key_logit(best) - lse;
+            if (o.draft_ids) o.draft_ids[out] = idx;
+        } else {   // fewer than k candidates exist only if a wait ran out upstream
+            o.target_ids[out] = -1;
+            o.logprobs[out] = -INFINITY;
+            if (o.draft_ids) o.draft_ids[out] = -1;
+        }
+    });
     if (lane == 0 && o.lse) o.lse[m] = lse;
 }
 
@@ -290,36 +367,57 @@ __device__ inline bool publish_and_check_last(WsHeader* hdr, int* smem_flag) {
 // of rows are brought into shared memory with one bulk copy per CTA record block (P copies in
 // flight at once: one L2 round trip per batch), then each warp merges one row at a time.
 //   stage_base/stage_bytes: shared memory the CTA no longer uses, 16-byte aligned, at least
-//                           P * (KS * 8 + 16) bytes;  bar: an initialised mbarrier (count 1), phase 0.
+//                           P * (KS * 8 + 16) + (warps of the CTA) * 2048 bytes;
+//   bar: an initialised mbarrier (count 1), phase 0.
 // Must be called by all threads of the CTA.
 __device__ inline void merge_rows(const HeadOut& o, int P, int m_begin, int m_count,
                                   unsigned char* stage_base, size_t stage_bytes, uint32_t bar) {
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
     const int KS = ws_slots(o.k), M = o.M;
-    int batch = (int)((stage_bytes / P - 16) / ((size_t)KS * 8));
+    // the tail of the region holds one candidate buffer per warp (warp_select_topk)
+    const size_t cand_bytes = (size_t)nwarps * kMergeCand * 8;
+    unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(stage_base + stage_bytes - cand_bytes) +
+                               (size_t)warp * kMergeCand;
+    stage_bytes -= cand_bytes;
+    const int pitch = ws_pitch(M, o.k);
+    unsigned long long* stage = reinterpret_cast<unsigned long long*>(stage_base);
+    const size_t all_bytes = (size_t)P * pitch * 8;
+    const bool one_copy = m_begin == 0 && m_count == M && all_bytes <= stage_bytes && all_bytes < (1u << 20);
+    int batch = one_copy ? m_count : (int)((stage_bytes / P - 16) / ((size_t)KS * 8));
     const int tx_cap = (int)(((1u << 20) - 16) / ((size_t)P * KS * 8));     // mbarrier byte-count limit
-    if (batch > tx_cap) batch = tx_cap;
+    if (!one_copy && batch > tx_cap) batch = tx_cap;
     if (batch > m_count) batch = m_count;
     if (batch < 1) batch = 1;
-    unsigned long long* stage = reinterpret_cast<unsigned long long*>(stage_base);
     fence_proxy_async();          // shared memory last touched by ordinary loads/stores is reused by bulk copies
     __syncthreads();
     uint32_t phase = 0;
     for (int b0 = 0; b0 < m_count; b0 += batch, phase ^= 1u) {
         const int nb = min(batch, m_count - b0);
-        int stride = nb * KS;                                  // u64 units between CTA record blocks
-        if (((stride >> 1) & 1) == 0) stride += 2;             // odd multiple of 16 bytes: at most 2-way bank conflicts
-        const uint32_t bytes = (uint32_t)nb * KS * 8;
-        if (threadIdx.x == 0) mbar_arrive_expect_tx(bar, bytes * (uint32_t)P);
-        __syncthreads();
-        for (int p = threadIdx.x; p < P; p += blockDim.x)
-            bulk_g2s(smem_u32(stage + (size_t)p * stride), o.recs + ((size_t)p * M + m_begin + b0) * KS, bytes, bar);
+        int stride;                                            // u64 units between CTA record blocks in shared memory
+        if (one_copy) {
+            // every CTA's records for all rows, padding included, are one contiguous block: a single copy
+            stride = pitch;
+            if (threadIdx.x == 0) {
+                mbar_arrive_expect_tx(bar, (uint32_t)all_bytes);
+                bulk_g2s(smem_u32(stage), o.recs, (uint32_t)all_bytes, bar);
+            }
+        } else {
+            stride = nb * KS;
+            if (((stride >> 1) & 1) == 0) stride += 2;         // odd multiple of 16 bytes: at most 2-way bank conflicts
+            const uint32_t bytes = (uint32_t)nb * KS * 8;
+            // The phase needs thread 0's arrival as well as all the bytes, so copies that land before the
+            // byte count is posted cannot complete it early: no barrier between posting and issuing.
+            if (threadIdx.x == 0) mbar_arrive_expect_tx(bar, bytes * (uint32_t)P);
+            for (int p = threadIdx.x; p < P; p += blockDim.x)
+                bulk_g2s(smem_u32(stage + (size_t)p * stride), VT_REC(o, p, m_begin + b0), bytes, bar);
+        }
         if (!mbar_wait(bar, phase)) {
             atomicOr(&o.hdr->status, kStatusTimeout);
             break;
         }
-        for (int r = warp; r < nb; r += nwarps) merge_row_final(o, P, m_begin + b0 + r, stage + (size_t)r * KS, stride);
+        for (int r = warp; r < nb; r += nwarps)
+            merge_row_final(o, P, m_begin + b0 + r, stage + (size_t)r * KS, stride, cbuf);
         __syncthreads();
     }
 }

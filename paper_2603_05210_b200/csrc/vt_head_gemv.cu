@@ -35,7 +35,7 @@ struct GemvParams {
     int n_stages;            // multiple of n_cons, so a stage is always consumed by the same warp
     int n_cons;              // consumer warps that take tiles (<= kGemvConsumers)
     uint32_t stage_bytes;
-    uint32_t h_off, list_off, bar_off, total_smem;
+    uint32_t h_off, list_off, fold_off, bar_off, total_smem;   // fold_off: candidate buffers of the per-row fold
 };
 
 // Folds NV per-lane values over the 32 lanes of a warp with NV-1 + log2(32/NV) shuffles.
@@ -216,11 +216,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         const unsigned long long* rec0 = lists + (size_t)m * KS;
         const int stride = MP * KS;
         const float2 ms = warp_merge_ms(rec0, stride, P1, k);
-        unsigned long long* dst = p.out.recs + ((size_t)cta * M + p.m_begin + m) * KS;
-        unsigned long long mine[2];
-        warp_merge_lists(rec0, stride, P1, k, mine);
-        if (lane < k) dst[lane] = mine[0];
-        if (lane + 32 < k) dst[lane + 32] = mine[1];
+        unsigned long long* dst = VT_REC(p.out, cta, p.m_begin + m);
+        unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(smem + p.fold_off) + (size_t)warp * kMergeCand;
+        warp_select_topk(rec0, stride, P1, k, cbuf, [&](int j, unsigned long long best) { dst[j] = best; });
         if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
     }
 
@@ -280,9 +278,13 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.stage_bytes = (uint32_t)sr * c.d * 2;
         const size_t h_bytes = ((size_t)MP * c.d * 2 + 127) & ~(size_t)127;
         const size_t list_bytes = ((size_t)kGemvConsumers * kGemvR * MP * KS * 8 + 127) & ~(size_t)127;
-        const size_t merge_bytes = (size_t)grid * (KS * 8 + 16);
+        const size_t cand_bytes = (size_t)kGemvWarps * kMergeCand * 8;
+        size_t merge_bytes = (size_t)grid * (KS * 8 + 16) + cand_bytes;            // one row per batch at least
+        const size_t one_copy = (size_t)grid * ws_pitch(c.out.M, c.out.k) * 8 + cand_bytes;   // all rows in one copy
+        if (c.out.fused_merge && one_copy <= 128 * 1024) merge_bytes = std::max(merge_bytes, one_copy);
         const size_t bar_bytes = (size_t)(2 * 32 + 1) * 8 + 16;
-        const size_t fixed = h_bytes + list_bytes + bar_bytes;
+        const size_t fold_bytes = (size_t)kGemvMaxM * kMergeCand * 8;
+        const size_t fixed = h_bytes + list_bytes + fold_bytes + bar_bytes;
         if (fixed + 2 * (size_t)p.stage_bytes > (size_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
         int S = (int)std::min<size_t>(32, ((size_t)kMaxDynSmem - fixed) / p.stage_bytes);
         p.n_cons = std::min(kGemvConsumers, S);
@@ -293,6 +295,8 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
         off += h_bytes;
         p.list_off = (uint32_t)off;
         off += list_bytes;
+        p.fold_off = (uint32_t)off;
+        off += fold_bytes;
         if (off < merge_bytes) off = (merge_bytes + 127) & ~(size_t)127;   // merge staging reuses [0, bar_off)
         p.bar_off = (uint32_t)off;
         p.total_smem = (uint32_t)(off + bar_bytes);

@@ -381,12 +381,12 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         }
         // records: the row's list is contiguous in shared memory, so k lanes copy it out together
         for (int row = 0; row < rows_here; ++row) {
-            unsigned long long* rec = p.out.recs + ((size_t)cta * M + p.m_begin + warp * 32 + row) * ws_slots(k);
+            unsigned long long* rec = VT_REC(p.out, cta, p.m_begin + warp * 32 + row);
             for (int j = lane; j < k; j += 32) rec[j] = lists[(size_t)row * k + j];
         }
         if (live) {
             const float2 ms = ms_s[warp * 32 + lane];
-            p.out.recs[((size_t)cta * M + p.m_begin + m_local) * ws_slots(k) + k] = pack_ms(ms.x, ms.y);
+            VT_REC(p.out, cta, p.m_begin + m_local)[k] = pack_ms(ms.x, ms.y);
         }
     } else if (team_mode && warp != 6) {
         // ------------------------------------------------------------------ selection helpers (warps 1-3, 7-11)
@@ -546,7 +546,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         const size_t list_bytes = (((size_t)epi_warps * 32 * c.out.k * 8 + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K) * 8 +
                                     (size_t)epi_warps * 32 * 12 + (size_t)epi_warps * p.tile_floats * 4) + 127) & ~(size_t)127;
         const size_t bar_bytes = (size_t)(2 * kMaxStages + 9) * 8 + 16;  // sized for the largest stage count
-        const size_t merge_bytes = (size_t)grid * (ws_slots(c.out.k) * 8 + 16);
+        const size_t merge_bytes = (size_t)grid * (ws_slots(c.out.k) * 8 + 16) + (size_t)(kMmaThreads / 32) * kMergeCand * 8;
         // Layout from the 1024-aligned base: ring | resident h | 16 KB the MMA may read past the last A block
         // (it always reads 128 A rows) | lists | barriers.  The pad is never written.
         const size_t fixed = 1024 + (p.h_resident ? h_bytes : 0) + 16384 + list_bytes + bar_bytes + 256;

@@ -23,10 +23,12 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const HeadOut o, i
 
 vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st) {
     const int KS = ws_slots(o.k);
+    const size_t cand = (size_t)(kMergeThreads / 32) * kMergeCand * 8;
     const size_t one_row = (size_t)P * (KS * 8 + 16);
     size_t want = (size_t)P * ((size_t)kMergeRowsPerCta * KS * 8 + 16);
     const size_t cap = 160 * 1024;
     if (want > cap) want = std::max(one_row, cap / one_row * one_row);
+    want += cand;
     if (want > (size_t)kMaxDynSmem - 1024) return VT_ERR_UNSUPPORTED;
     static int configured_device = -1;
     int dev = 0;
