@@ -117,24 +117,51 @@ def to_dev(a, torch, dtype=None):
     return t.view(dtype) if dtype is not None else t
 
 
-def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0):
-    """CUDA-event time of `steps` back-to-back calls rotating over W_copies; returns ms total."""
+GRAPH_CALLS = 120     # calls per captured CUDA graph (a multiple of every copy count the bench uses: 2..6, 8, 10, 12...)
+
+
+def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=True):
+    """CUDA-event time of exactly `steps` back-to-back calls rotating over W_copies; returns (ms total, launches/call).
+
+    With use_graph the calls are replayed from a captured CUDA graph of GRAPH_CALLS calls (plus directly
+    launched calls for the remainder), the way a serving loop would issue them; otherwise every call goes
+    through the Python binding.  Either way each call is a separate kernel launch on the stream.
+    """
     M = h.shape[0]
     ws = vt.new_workspace(vt.vt_workspace_bytes(M, k))
     tid = torch.empty((M, k), dtype=torch.int32, device="cuda")
     lp = torch.empty((M, k), dtype=torch.float32, device="cuda")
     n = len(W_copies)
-    for i in range(warmup):
+
+    def call(i):
         vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+
+    for i in range(warmup):
+        call(i)
+    launches = vt.vt_last_launch_count()
+    graph = None
+    n_replay = steps // GRAPH_CALLS if use_graph else 0
+    if n_replay > 0:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(GRAPH_CALLS):
+                    call(i)
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()                                   # one untimed replay: graph upload
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     e0.record()
-    for i in range(steps):
-        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+    for _ in range(n_replay):
+        graph.replay()
+    for i in range(steps - n_replay * GRAPH_CALLS):
+        call(i)
     e1.record()
     torch.cuda.synchronize()
     assert vt.vt_last_status(ws) == vt.VT_OK, "a device-side wait ran out during the timed region"
-    return e0.elapsed_time(e1), vt.vt_last_launch_count()
+    return e0.elapsed_time(e1), launches
 
 
 def n_copies_for_cold(bytes_per_copy, l2_bytes, free_bytes):
@@ -200,7 +227,7 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    ms, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup)
+    ms, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup, use_graph=not args.no_graph)
     clocks = sampler.stop()
     ms = max_over_ranks(ms, dist, "cuda")
     if dist is not None:
@@ -232,6 +259,8 @@ def run_ours(args):
         "config": {"workload": WORKLOAD_NAME, "cold": f"calls rotate over {nc} copies of W_trim "
                    f"({nc * W_trim.numel() * 2 / 1e6:.0f} MB >= 4x L2 of {l2 / 1e6:.0f} MB): inputs larger than L2",
                    "step": "one vt_draft_head call (contraction + top-k + log-softmax + remap, one launch)",
+                   "launch": "eager calls through the binding" if args.no_graph or args.steps < GRAPH_CALLS
+                   else f"CUDA-graph replay of {GRAPH_CALLS}-call graphs (one kernel launch per call)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "calls_per_s": round(1e6 / value, 1)},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
@@ -250,7 +279,7 @@ def run_ours(args):
 
     if rank == 0 and world == 1:
         if not args.no_curve:
-            line["curve"] = latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs)
+            line["curve"] = latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, not args.no_graph)
         line["cpu_baseline"] = cpu_baseline(case)
     if rank == 0:
         print(json.dumps(line))
@@ -258,7 +287,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs):
+def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, use_graph=True):
     """us/call and roofline fraction over V_trim x M at d=4096 (the measured latency-vs-vocabulary curve)."""
     d, k = case.d, 8
     order = ranking[0]
@@ -272,8 +301,8 @@ def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs):
         for M in CURVE_M:
             h = to_dev(inputs.hidden_states_bf16(M, d, 77 + M).view(np.int16), torch, torch.bfloat16)
             kk = min(k, Vt)
-            steps = 400 if Vt <= 32000 else 100
-            ms, _ = time_head(vt, torch, h, copies, keep, kk, steps, 20)
+            steps = 480 if Vt <= 32000 else 120
+            ms, _ = time_head(vt, torch, h, copies, keep, kk, steps, 20, use_graph=use_graph)
             us = ms * 1000.0 / steps
             gbs = head_bytes(d, Vt, M, kk) / (us * 1e-6) / 1e9
             out.append({"V_trim": Vt, "M": M, "us_per_call": round(us, 2), "GBs": round(gbs, 1),
@@ -349,6 +378,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-curve", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every timed call through the binding instead of a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -31,7 +31,13 @@ struct MmaParams {
     HeadOut out;
     int m_begin, m_count;     // draft rows of this pass
     int d;
-    int NT;                   // vocabulary rows per tile (multiple of 16, <= 256)
+    int NT;                   // vocabulary rows per main tile (multiple of 16, <= 256)
+    int n_main;               // main tiles a CTA with the most rows has
+    int NT_tail;              // rows of the short tile that follows them (0: none); its epilogue is the only one
+                              // that cannot hide behind the weight stream, so it is kept short
+    uint32_t idesc_tail;
+    int kb_tail;              // k-blocks per stage and bytes per k-block while the tail tile streams
+    uint32_t blk_tail;
     int nk;                   // 64-column k-blocks per tile
     int kb_per_stage;         // k-blocks one ring stage holds (one barrier hand-over per stage)
     uint32_t blk_bytes;       // bytes of one k-block in a stage: (A slot +) B slot, multiple of 1024
@@ -92,7 +98,6 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-constexpr int kHelpers = 8;                   // warps 1-3 and 7-11 share the top-k selection when one warp owns all draft rows
 constexpr int kMaxBatchCols = 256;            // vocabulary columns the top-k selection takes at a time
 
 // Top-k update of one draft row by a whole warp.  `vals` is the row's logits for `ncols` consecutive
@@ -167,7 +172,8 @@ __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, 
 // through shared memory so that a whole warp works on one draft row at a time (warp_topk_update), which
 // keeps all 32 lanes busy when there are only a few draft rows.
 __global__ void __launch_bounds__(kMmaThreads, 1)
-head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
+head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWt,
+                const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -179,7 +185,11 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
     const int row_begin = (int)((long long)cta * Vt / G);
     const int row_end = (int)((long long)(cta + 1) * Vt / G);
     const int nrows = row_end - row_begin;
-    const int ntiles = (nrows + NT - 1) / NT;
+    // tiles of this CTA: up to n_main tiles of NT rows, then (if rows remain) one tile of NT_tail rows
+    const int main_here = min(p.n_main, (nrows + NT - 1) / NT);
+    const bool tail_here = p.NT_tail > 0 && nrows > p.n_main * NT;
+    const int ntiles = main_here + (tail_here ? 1 : 0);
+    auto tile_rows = [&](int t) { return (tail_here && t == ntiles - 1) ? p.NT_tail : NT; };
 
     unsigned long long* epi = reinterpret_cast<unsigned long long*>(smem + p.list_off);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
@@ -204,15 +214,14 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
         mbar_init(bar_drain, 1);
         mbar_init(bar_merge, 1);
         mbar_init(bar_h, 1);
-        mbar_init(bar_sel_ready, 1);
-        mbar_init(bar_sel_done, kHelpers);
+        mbar_init(bar_sel_ready, n_epi_warps);
+        mbar_init(bar_sel_done, n_epi_warps + (4 - n_epi_warps) + (kMmaThreads / 32 - 7));
         *abort_flag = 0;
         fence_mbar_init();
     }
     // epilogue scratch: lists [warps * 32][k] keys | candidate staging per warp | transpose buffer per warp
     for (int i = tid; i < n_epi_warps * 32 * k; i += blockDim.x) epi[i] = 0ull;
-    const bool team_mode = n_epi_warps == 1;       // all draft rows in warp 0: idle warps help with the selection
-    const int n_cbuf = team_mode ? 1 + kHelpers : n_epi_warps;
+    const int n_cbuf = 4 + (kMmaThreads / 32 - 7);  // one candidate buffer per team member (readers and helpers)
     unsigned long long* cands = epi + (size_t)n_epi_warps * 32 * k;
     float* thr_s = reinterpret_cast<float*>(cands + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K));   // [warps * 32]
     float2* ms_s = reinterpret_cast<float2*>(thr_s + n_epi_warps * 32);                               // [warps * 32]
@@ -255,19 +264,24 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * NT;
-                for (int ks = 0; ks < nk; ks += p.kb_per_stage) {
+                const bool is_tail = tail_here && t == ntiles - 1;
+                const CUtensorMap* mapW = is_tail ? &tmWt : &tmW;
+                const uint32_t b_tx = (uint32_t)tile_rows(t) * 128u;
+                const int kbs = is_tail ? p.kb_tail : p.kb_per_stage;
+                const uint32_t blk = is_tail ? p.blk_tail : p.blk_bytes;
+                for (int ks = 0; ks < nk; ks += kbs) {
                     if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
-                    const int nb = min(p.kb_per_stage, nk - ks);
+                    const int nb = min(kbs, nk - ks);
                     const uint32_t bar = bar_full + 8u * s;
-                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (p.h_resident ? p.b_tx : p.a_tx + p.b_tx));
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (p.h_resident ? b_tx : p.a_tx + b_tx));
                     for (int kb = 0; kb < nb; ++kb) {
-                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
+                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * blk;
                         if (p.h_resident) {
-                            tma_load_2d(dst, &tmW, (ks + kb) * kBoxK, row0, bar);
+                            tma_load_2d(dst, mapW, (ks + kb) * kBoxK, row0, bar);
                         } else {
                             tma_load_2d(dst, &tmH, (ks + kb) * kBoxK, p.m_begin, bar);
-                            tma_load_2d(dst + p.a_slot, &tmW, (ks + kb) * kBoxK, row0, bar);
+                            tma_load_2d(dst + p.a_slot, mapW, (ks + kb) * kBoxK, row0, bar);
                         }
                     }
                     ++issued;
@@ -289,26 +303,30 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             if (p.h_resident && ntiles > 0 && !mbar_wait(bar_h, 0u)) { fail(); ok = false; }
             const uint64_t desc0 = smem_desc_sw128(base);                      // descriptor of the ring's first byte
             const uint64_t h_desc0 = smem_desc_sw128(base + p.h_off);
-            const uint32_t stage_units = p.stage_bytes >> 4, a_units = p.a_slot >> 4, blk_units = p.blk_bytes >> 4;
+            const uint32_t stage_units = p.stage_bytes >> 4, a_units = p.a_slot >> 4;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
-                for (int ks = 0; ks < nk; ks += p.kb_per_stage) {
+                const bool is_tail = tail_here && t == ntiles - 1;
+                const uint32_t idesc = is_tail ? p.idesc_tail : p.idesc;
+                const int kbs = is_tail ? p.kb_tail : p.kb_per_stage;
+                const uint32_t blk_units = (is_tail ? p.blk_tail : p.blk_bytes) >> 4;
+                for (int ks = 0; ks < nk; ks += kbs) {
                     if (!mbar_wait(bar_full + 8u * s, phase)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
-                    const int nb = min(p.kb_per_stage, nk - ks);
+                    const int nb = min(kbs, nk - ks);
                     for (int kb = 0; kb < nb; ++kb) {
                         const uint64_t blk_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * blk_units);
                         const uint64_t a_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)(ks + kb) * a_units) : blk_desc;
                         const uint64_t b_desc = p.h_resident ? blk_desc : blk_desc + a_units;
                         // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
-                        tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (ks | kb) != 0);
+                        tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
                     }
                     tc_commit(bar_empty + 8u * s);
                     if (++s == S) { s = 0; phase ^= 1u; }
@@ -320,105 +338,95 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 (void)mbar_wait(bar_drain, 0u);
             }
         }
-    } else if (warp < n_epi_warps) {
-        // ------------------------------------------------------------------ epilogue: TMEM reader
+    } else if (warp < n_epi_warps || warp >= 7 || warp < 4) {
+        // ------------------------------------------------------------------ epilogue team
+        // Readers (warps 0 .. n_epi_warps-1) own a quarter of the TMEM lanes each and turn their draft rows'
+        // logits into the transpose buffers; then every team member - the readers and the otherwise idle
+        // warps (the other warps below 4, and warps 7-11) - takes every team-th draft row of the batch.
+        // Helpers replay the readers' batch sequence, which depends only on the tile geometry.
+        const bool reader = warp < n_epi_warps;
+        const int n_help = (4 - n_epi_warps) + (kMmaThreads / 32 - 7);
+        const int team = n_epi_warps + n_help;
+        const int member = reader ? warp : (warp < 4 ? warp : n_epi_warps + (4 - n_epi_warps) + (warp - 7));
         const int m_local = warp * 32 + lane;
-        const bool live = m_local < p.m_count;
-        const int rows_here = min(32, p.m_count - warp * 32);          // live draft rows of this warp
+        const bool live = reader && m_local < p.m_count;
         const int EB = p.batch_cols, EBP = EB + 1;                     // odd row pitch: conflict-free both ways
-        float* tbuf = tiles + (size_t)warp * p.tile_floats;            // tbuf[row * EBP + column in batch]
-        unsigned long long* cbuf = cands + (size_t)warp * (kMaxBatchCols + VT_MAX_K);
-        unsigned long long* lists = epi + (size_t)warp * 32 * k;       // lists[row * k + j]
+        float* my_tbuf = tiles + (size_t)warp * p.tile_floats;         // reader: tbuf[row * EBP + column in batch]
+        unsigned long long* cbuf = cands + (size_t)member * (kMaxBatchCols + VT_MAX_K);
         uint32_t batch_no = 0;
+        bool ok = true;
 
-        for (int t = 0; t < ntiles; ++t) {
+        for (int t = 0; t < ntiles && ok; ++t) {
             const int buf = t & 1;
-            if (!mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u)) { fail(); break; }
-            if (*abort_flag) break;
-            tc_fence_after();
+            if (reader) {
+                if (!mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u)) { fail(); break; }
+                if (*abort_flag) break;
+                tc_fence_after();
+            }
             const int row0 = row_begin + t * NT;
-            const int ncols = min(NT, row_end - row0);
+            const int ncols = min(tile_rows(t), row_end - row0);
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kAccStride);
             for (int c0 = 0; c0 < ncols; c0 += 32) {
-                uint32_t r[32];
-                tc_ld32(taddr + (uint32_t)c0, r);
-                tc_wait_ld();
                 const int nv = min(32, ncols - c0);
                 const int cb = c0 % EB;                                // column of this chunk inside the batch
-                // lane = draft row: the chunk goes to the transpose buffer (columns past the CTA's rows are not its logits)
-                if (live) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) tbuf[lane * EBP + cb + c] = c < nv ? __uint_as_float(r[c]) : -INFINITY;
-                    if (p.out.logits) {
-                        float* dst = p.out.logits + (size_t)(p.m_begin + m_local) * Vt + row0 + c0;
+                const bool tile_end = c0 + 32 >= ncols;
+                if (reader) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + (uint32_t)c0, r);
+                    tc_wait_ld();
+                    // lane = draft row; columns past the CTA's rows are not its logits
+                    if (live) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c < nv) dst[c] = __uint_as_float(r[c]);
+                            my_tbuf[lane * EBP + cb + c] = c < nv ? __uint_as_float(r[c]) : -INFINITY;
+                        if (p.out.logits) {
+                            float* dst = p.out.logits + (size_t)(p.m_begin + m_local) * Vt + row0 + c0;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c < nv) dst[c] = __uint_as_float(r[c]);
+                        }
                     }
                 }
-                // a full batch (or the tile's last chunk): one warp per draft row takes it from here
-                if (cb + 32 >= EB || c0 + 32 >= ncols) {
-                    if (c0 + 32 >= ncols) {          // TMEM is read out: the MMAs of the tile after next may start
+                if (!(cb + 32 >= EB || tile_end)) continue;
+                // a batch is complete (EB columns, or the tile's last chunk)
+                if (reader) {
+                    if (tile_end) {                  // TMEM is read out: the MMAs of the tile after next may start
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
                     }
                     __syncwarp();
-                    if (team_mode && lane == 0) mbar_arrive(bar_sel_ready);
-                    const int bvalid = min(min(cb + 32, EB), ncols - (c0 - cb));   // valid columns of the batch
-                    const int bcol0 = row0 + c0 - cb;                              // vocabulary row of its first column
-                    const int team = team_mode ? 1 + kHelpers : 1;
-                    for (int row = 0; row < rows_here; row += team) {
-                        const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
-                                                          thr_s[warp * 32 + row], cbuf, ms_s + warp * 32 + row, lane);
-                        if (lane == 0) thr_s[warp * 32 + row] = t2;
-                    }
-                    __syncwarp();
-                    if (team_mode && !mbar_wait(bar_sel_done, batch_no & 1u)) { fail(); break; }
-                    ++batch_no;
+                    if (lane == 0) mbar_arrive(bar_sel_ready);
                 }
+                if (!mbar_wait(bar_sel_ready, batch_no & 1u)) { fail(); ok = false; break; }
+                if (*abort_flag) { ok = false; break; }
+                const int bvalid = min(min(cb + 32, EB), ncols - (c0 - cb));   // valid columns of the batch
+                const int bcol0 = row0 + c0 - cb;                              // vocabulary row of its first column
+                for (int m = member; m < p.m_count; m += team) {
+                    const float* vals = tiles + (size_t)(m >> 5) * p.tile_floats + (size_t)(m & 31) * EBP;
+                    const float t2 = warp_topk_update(vals, bvalid, bcol0, epi + (size_t)m * k, k, thr_s[m], cbuf,
+                                                      ms_s + m, lane);
+                    if (lane == 0) thr_s[m] = t2;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sel_done);
+                // the transpose buffers are rewritten only after the whole team is done with them
+                if (reader && !mbar_wait(bar_sel_done, batch_no & 1u)) { fail(); ok = false; break; }
+                ++batch_no;
             }
         }
-        // records: the row's list is contiguous in shared memory, so k lanes copy it out together
-        for (int row = 0; row < rows_here; ++row) {
-            unsigned long long* rec = VT_REC(p.out, cta, p.m_begin + warp * 32 + row);
-            for (int j = lane; j < k; j += 32) rec[j] = lists[(size_t)row * k + j];
-        }
-        if (live) {
-            const float2 ms = ms_s[warp * 32 + lane];
-            VT_REC(p.out, cta, p.m_begin + m_local)[k] = pack_ms(ms.x, ms.y);
-        }
-    } else if (team_mode && warp != 6) {
-        // ------------------------------------------------------------------ selection helpers (warps 1-3, 7-11)
-        // They replay the reader's batch sequence (it depends only on the tile geometry) and take every
-        // (1 + kHelpers)-th draft row of each batch.
-        const int member = warp < 4 ? warp : warp - 3;                 // 1..kHelpers
-        const int rows_here = p.m_count;
-        const int EB = p.batch_cols, EBP = EB + 1;
-        const float* tbuf = tiles;
-        unsigned long long* cbuf = cands + (size_t)member * (kMaxBatchCols + VT_MAX_K);
-        unsigned long long* lists = epi;
-        uint32_t batch_no = 0;
-        bool ok = true;
-        for (int t = 0; t < ntiles && ok; ++t) {
-            const int row0 = row_begin + t * NT;
-            const int ncols = min(NT, row_end - row0);
-            for (int c0 = 0; c0 < ncols; c0 += 32) {
-                const int cb = c0 % EB;
-                if (cb + 32 >= EB || c0 + 32 >= ncols) {
-                    if (!mbar_wait(bar_sel_ready, batch_no & 1u)) { fail(); ok = false; break; }
-                    if (*abort_flag) { ok = false; break; }
-                    const int bvalid = min(min(cb + 32, EB), ncols - (c0 - cb));
-                    const int bcol0 = row0 + c0 - cb;
-                    for (int row = member; row < rows_here; row += 1 + kHelpers) {
-                        const float t2 = warp_topk_update(tbuf + row * EBP, bvalid, bcol0, lists + (size_t)row * k, k,
-                                                          thr_s[row], cbuf, ms_s + row, lane);
-                        if (lane == 0) thr_s[row] = t2;
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_sel_done);
-                    ++batch_no;
-                }
+        if (reader) {
+            // records: a row's list is contiguous in shared memory, so k lanes copy it out together.  Rows
+            // another member kept are visible: its arrival on bar_sel_done released them.
+            const int rows_here = min(32, p.m_count - warp * 32);
+            for (int row = 0; row < rows_here; ++row) {
+                const int m = warp * 32 + row;
+                unsigned long long* rec = VT_REC(p.out, cta, p.m_begin + m);
+                for (int j = lane; j < k; j += 32) rec[j] = epi[(size_t)m * k + j];
+            }
+            if (live) {
+                const float2 ms = ms_s[m_local];
+                VT_REC(p.out, cta, p.m_begin + m_local)[k] = pack_ms(ms.x, ms.y);
             }
         }
     }
@@ -470,17 +478,28 @@ static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, in
     return cr == CUDA_SUCCESS ? VT_OK : driver_fail((int)cr);
 }
 
-// Tile height: a multiple of 16 in [16, 256] that covers ceil(Vt / grid) rows with the least padding (rows
-// past the CTA's range that a tile still loads are wasted HBM traffic), preferring taller tiles among
-// equals: fewer accumulator hand-overs and fewer selection batches per draft row.
-static int choose_tile_rows(int rows_per_cta) {
-    int best = 16, best_pad = 1 << 30;
+// Tiling of the most rows a CTA owns: n_main tiles of NT rows plus, optionally, one short tail tile whose
+// epilogue (the only one nothing streams behind) would be shorter.  Measured on B200 a 48- or 64-row tail
+// streams too slowly to pay for itself (an MMA costs 45 cycles however few rows it covers, and every ring
+// stage a barrier hand-over), so kMaxTailRows is 0 and the search only picks the main tile: the multiple
+// of 16 that covers the rows with the least padding - rows a tile loads past the CTA's range are wasted
+// HBM traffic - preferring taller tiles among equals.
+struct Tiling { int NT, n_main, NT_tail; };
+constexpr int kMaxTailRows = 0;
+static Tiling choose_tiling(int rows) {
+    Tiling best{16, (rows + 15) / 16, 0};
+    int best_cost = 1 << 30;
     for (int nt = 16; nt <= 256; nt += 16) {
-        const int tiles = (rows_per_cta + nt - 1) / nt;
-        const int pad = tiles * nt - rows_per_cta;
-        if (pad < best_pad || (pad == best_pad && nt > best)) {
-            best = nt;
-            best_pad = pad;
+        for (int tail = 0; tail <= kMaxTailRows; tail += 16) {
+            if (tail > 0 && (tail < 48 || tail >= rows)) continue;
+            const int n_main = (rows - tail + nt - 1) / nt;
+            if (tail > 0 && rows <= n_main * nt) continue;          // the tail would be empty
+            const int pad = n_main * nt + tail - rows;
+            const int cost = pad * 1024 + (tail > 0 ? tail : 256 - nt);          // least padding, then the taller tile
+            if (cost < best_cost) {
+                best_cost = cost;
+                best = Tiling{nt, n_main, tail};
+            }
         }
     }
     return best;
@@ -493,7 +512,8 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
     const int rows_per_cta = (c.Vt + grid - 1) / grid;
-    const int NT = choose_tile_rows(rows_per_cta);
+    const Tiling tiling = choose_tiling(rows_per_cta);
+    const int NT = tiling.NT;
 
     static int configured_device = -1;
     int dev = 0;
@@ -507,6 +527,11 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     CUtensorMap tmW;
     r = make_map(&tmW, c.W, c.Vt, c.d, NT);
     if (r != VT_OK) return r;
+    CUtensorMap tmWt = tmW;
+    if (tiling.NT_tail > 0) {
+        r = make_map(&tmWt, c.W, c.Vt, c.d, tiling.NT_tail);
+        if (r != VT_OK) return r;
+    }
 
     for (int m0 = 0; m0 < c.M; m0 += 128) {
         const int mc = std::min(128, c.M - m0);
@@ -520,6 +545,8 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.m_count = mc;
         p.d = c.d;
         p.NT = NT;
+        p.n_main = tiling.n_main;
+        p.NT_tail = tiling.NT_tail;
         p.nk = (c.d + kBoxK - 1) / kBoxK;
         p.a_tx = (uint32_t)mc * 128u;
         p.b_tx = (uint32_t)NT * 128u;
@@ -532,8 +559,11 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.kb_per_stage = std::max(1, std::min(4, (int)((28 * 1024 + p.blk_bytes / 2) / p.blk_bytes)));
         p.kb_per_stage = std::min(p.kb_per_stage, p.nk);
         p.stage_bytes = p.blk_bytes * p.kb_per_stage;
+        p.blk_tail = (p.h_resident ? 0u : p.a_slot) + (((uint32_t)tiling.NT_tail * 128u + 1023u) & ~1023u);
+        p.kb_tail = tiling.NT_tail > 0 ? std::max(1, std::min(p.nk, (int)(p.stage_bytes / p.blk_tail))) : 1;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        p.idesc_tail = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tiling.NT_tail >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // epilogue scratch: lists, candidate staging and a transpose buffer per epilogue warp; the fewer draft
         // rows a warp has, the more columns it can afford to select from at a time
         const int epi_warps = (mc + 31) / 32;
@@ -542,7 +572,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         while (batch > 32 && (size_t)rows_w * (batch + 1) * 4 > 17 * 1024) batch -= 32;
         p.batch_cols = batch;
         p.tile_floats = (uint32_t)(rows_w * (batch + 1));
-        const int n_cbuf = epi_warps == 1 ? 1 + kHelpers : epi_warps;
+        const int n_cbuf = 4 + (kMmaThreads / 32 - 7);
         const size_t list_bytes = (((size_t)epi_warps * 32 * c.out.k * 8 + (size_t)n_cbuf * (kMaxBatchCols + VT_MAX_K) * 8 +
                                     (size_t)epi_warps * 32 * 12 + (size_t)epi_warps * p.tile_floats * 4) + 127) & ~(size_t)127;
         const size_t bar_bytes = (size_t)(2 * kMaxStages + 9) * 8 + 16;  // sized for the largest stage count
@@ -561,7 +591,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.bar_off = (uint32_t)((p.list_off + list_bytes + 127) & ~(size_t)127);
         p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
 
-        head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmH, p);
+        head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmWt, tmH, p);
         count_launch();
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e);
