@@ -104,8 +104,8 @@ constexpr int kMaxBatchCols = 256;            // vocabulary columns the top-k se
 // vocabulary columns (first column = vocabulary row `col0`), in shared memory; `list` is the row's k best
 // so far (descending keys, 0 = empty) and `tau` the logit of its k-th best (-inf while the list is not
 // full).  Lane L looks at columns L, L+32, ...
-//   1. bound: the 32 lanes form 8 groups of 4; the smallest of the 8 group maxima has at least 8 logits at
-//      or above it, so with k <= 8 nothing below it can be among the k best of these columns;
+//   1. bound: the 32 lanes form 8, 16 or 32 groups (whichever is >= k; k <= 32); the smallest group maximum
+//      has at least k logits at or above it, so nothing below it can be among the k best of these columns;
 //   2. the logits above tau (strictly: a later row loses a tie) and not below the bound are the candidates;
 //      a ballot per column group gives each its slot in `cbuf`, and the current list follows them;
 //   3. every entry of cbuf counts the entries larger than itself - its rank - and the entries of rank < k
@@ -137,12 +137,13 @@ __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, 
     }
     if (!__any_sync(0xFFFFFFFFu, lmax > tau)) return tau;
     float bound = -INFINITY;
-    if (k <= 8) {
-        float g = fmaxf(lmax, __shfl_xor_sync(0xFFFFFFFFu, lmax, 1));
-        g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
-        g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
-        g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 8));
-        bound = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 16));
+    if (k <= 32) {      // 8 groups of 4 lanes, 16 of 2 or 32 of 1: at least k group maxima, all distinct logits
+        float g = lmax;
+        if (k <= 16) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+        if (k <= 8) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, o));
+        bound = g;
     }
     int n = 0;
 #pragma unroll
@@ -487,9 +488,12 @@ static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, in
 struct Tiling { int NT, n_main, NT_tail; };
 constexpr int kMaxTailRows = 0;
 static Tiling choose_tiling(int rows) {
-    Tiling best{16, (rows + 15) / 16, 0};
+    // tiles below 96 rows only when the CTA has fewer rows than that: every ring stage costs a barrier
+    // hand-over and every MMA 45 cycles however few rows it covers
+    if (rows <= 96) return Tiling{((rows + 15) / 16) * 16, 1, 0};
+    Tiling best{256, (rows + 255) / 256, 0};
     int best_cost = 1 << 30;
-    for (int nt = 16; nt <= 256; nt += 16) {
+    for (int nt = 96; nt <= 256; nt += 16) {
         for (int tail = 0; tail <= kMaxTailRows; tail += 16) {
             if (tail > 0 && (tail < 48 || tail >= rows)) continue;
             const int n_main = (rows - tail + nt - 1) / nt;
