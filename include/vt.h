@@ -131,7 +131,8 @@ vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d
  * h_host (host [M, d] bf16, ideally pinned) is copied to the device, the head runs, and
  * target_ids_host / logprobs_host (host [M, k]) are copied back, all on `stream`; the call
  * SYNCHRONISES the stream before returning so the host outputs are valid.  W_trim and d2t
- * stay device-resident (they are model state, not per-step input).
+ * stay device-resident (they are model state, not per-step input).  Pinned (page-locked, mapped) output
+ * buffers are written by the kernel directly; pageable ones are filled by two copies after it.
  * workspace: dev, vt_host_workspace_bytes(M, d, k) bytes, initialised with vt_workspace_init. */
 size_t    vt_host_workspace_bytes(int M, int d, int k);
 vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32_t* d2t,

@@ -213,15 +213,31 @@ vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32
     vt_status r = check_head_args(h_dev, W_trim, d2t, M, d, V_trim, k, tid_dev, lp_dev, workspace, head_ws);
     if (r != VT_OK) return r;
     cudaStream_t st = (cudaStream_t)stream;
+    // Pinned host outputs are written by the merge directly (they are device-accessible under unified
+    // addressing): no device-to-host copies.  Pageable outputs go through the staging buffers.
+    int32_t* tid_out = tid_dev;
+    float* lp_out = lp_dev;
+    cudaPointerAttributes at_tid{}, at_lp{};
+    const bool direct = cudaPointerGetAttributes(&at_tid, target_ids_host) == cudaSuccess &&
+                        cudaPointerGetAttributes(&at_lp, logprobs_host) == cudaSuccess &&
+                        at_tid.type == cudaMemoryTypeHost && at_lp.type == cudaMemoryTypeHost &&
+                        at_tid.devicePointer && at_lp.devicePointer;
+    (void)cudaGetLastError();      // a pageable pointer makes the query fail on some drivers; that is not an error here
+    if (direct) {
+        tid_out = reinterpret_cast<int32_t*>(at_tid.devicePointer);
+        lp_out = reinterpret_cast<float*>(at_lp.devicePointer);
+    }
     cudaError_t e = cudaMemcpyAsync(h_dev, h_host, (size_t)M * d * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
-    HeadCall c{h_dev, W_trim, d, M, V_trim, make_out(d2t, M, V_trim, k, tid_dev, lp_dev, nullptr, nullptr, nullptr, workspace)};
+    HeadCall c{h_dev, W_trim, d, M, V_trim, make_out(d2t, M, V_trim, k, tid_out, lp_out, nullptr, nullptr, nullptr, workspace)};
     r = run_head(c, st, VT_PATH_AUTO);
     if (r != VT_OK) return r;
-    e = cudaMemcpyAsync(target_ids_host, tid_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaMemcpyAsync(logprobs_host, lp_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) return cuda_fail(e);
+    if (!direct) {
+        e = cudaMemcpyAsync(target_ids_host, tid_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaMemcpyAsync(logprobs_host, lp_dev, (size_t)M * k * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     e = cudaStreamSynchronize(st);
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
 }

@@ -199,13 +199,19 @@ def test_trimmed_head_equals_full_head_restricted(vt, oracle):
     assert np.array_equal(got_full["target_ids"][:, 0], np.argmax(oracle.logits(h, W_full), axis=1))
 
 
-def test_host_buffer_entry_point(vt, oracle):
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned", "pageable"])
+def test_host_buffer_entry_point(vt, oracle, pinned):
     M, d, Vt, k = 8, 1024, 3000, 8
     h, W, d2t = rand_case(M, d, Vt, seed=13)
     ws = vt.new_workspace(vt.vt_host_workspace_bytes(M, d, k))
-    h_host = torch.from_numpy(h.view(np.int16)).pin_memory()
-    tid = torch.empty((M, k), dtype=torch.int32).pin_memory()
-    lp = torch.empty((M, k), dtype=torch.float32).pin_memory()
-    vt.vt_draft_head_host(h_host, dev_bf16(W), dev_i32(d2t), k, tid, lp, ws)
+    h_host = torch.from_numpy(h.view(np.int16).copy())
+    tid = torch.full((M, k), -7, dtype=torch.int32)
+    lp = torch.full((M, k), float("nan"), dtype=torch.float32)
+    if pinned:      # pinned outputs are written by the kernel itself, pageable ones by copies after it
+        h_host, tid, lp = h_host.pin_memory(), tid.pin_memory(), lp.pin_memory()
+    Wd, d2td = dev_bf16(W), dev_i32(d2t)
     ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
-    parity.check_head({"target_ids": tid.numpy(), "logprobs": lp.numpy()}, ora, d2t, k)
+    for _ in range(2):
+        tid.fill_(-7)
+        vt.vt_draft_head_host(h_host, Wd, d2td, k, tid, lp, ws)
+        parity.check_head({"target_ids": tid.numpy().copy(), "logprobs": lp.numpy().copy()}, ora, d2t, k)
