@@ -1,0 +1,104 @@
+"""Pins for the selection oracle: the paper's printed numbers (Table 1, Section 2.6), exact rational brute force,
+closed forms and the limiting cases of the objective (Eq. 1-5)."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import vt_select_oracle as so
+from paper_2603_05210_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "table1_flops.txt")
+
+
+def golden():
+    out = {}
+    for line in open(GOLD):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+def test_table1_flops_and_shares_reproduce():
+    g = golden()
+    d, V = int(g["d"]), int(g["V"])
+    head = 2 * d * V
+    fusion = 2 * (3 * d) * d
+    assert head == 1_050_673_152 and round(head / 1e6, 1) == g["lm_head_mflop"]
+    assert round(fusion / 1e6, 1) == g["fusion_mflop"]
+    F_fixed = so.fixed_flops(d, g["attention_mflop"] * 1e6, g["feed_forward_mflop"] * 1e6)
+    total = F_fixed + head
+    assert abs(total / 1e6 - g["total_mflop"]) < 0.1        # the printed total adds the rounded entries (1637.9 vs 1637.84)
+    assert round(100 * head / total, 1) == g["lm_head_share_pct"]
+    assert round(100 * fusion / total, 1) == g["fusion_share_pct"]
+    assert round(100 * g["attention_mflop"] * 1e6 / total, 1) == g["attention_share_pct"]
+    assert round(100 * g["feed_forward_mflop"] * 1e6 / total, 1) == g["feed_forward_share_pct"]
+
+
+def test_eq3_worked_values_from_section_2_6():
+    g = golden()
+    d, V = int(g["d"]), int(g["V"])
+    F_fixed = so.fixed_flops(d, g["attention_mflop"] * 1e6, g["feed_forward_mflop"] * 1e6)
+    R = so.reduction(int(g["k_star"]), d, V, F_fixed)
+    assert abs(100 * float(R) - g["R_at_k_star_pct"]) < 0.05          # 57.5 % at k = 13,264
+    assert round(100 * float(so.reduction(0, d, V, F_fixed))) == g["R_max_pct"]   # "up to 64 %"
+    assert float(so.reduction(V, d, V, F_fixed)) == 0.0                # the untrimmed head saves nothing
+    ks = np.arange(1, V + 1)
+    Rk = so.reduction(ks, d, V, F_fixed)
+    assert np.all(np.diff(Rk) < 0)                                     # strictly decreasing, linear in k
+    assert np.allclose(np.diff(Rk), np.diff(Rk)[0], rtol=1e-6)
+
+
+def exact_curves(tokens, V, d, F_fixed, alpha):
+    f = [0] * V
+    for t in tokens:
+        f[t] += 1
+    order = sorted(range(V), key=lambda v: (-f[v], v))
+    total = sum(f)
+    cum, C, R, U = 0, [], [], []
+    for k in range(1, V + 1):
+        cum += f[order[k - 1]]
+        C.append(Fraction(cum, total))
+        R.append(1 - Fraction(F_fixed + 2 * d * k, F_fixed + 2 * d * V))
+        U.append(alpha * C[-1] + (1 - alpha) * R[-1])
+    return f, order, C, R, U
+
+
+@pytest.mark.parametrize("seed,alpha,c_min", [(0, Fraction(1, 2), Fraction(9, 10)), (1, Fraction(7, 10), Fraction(1, 2)),
+                                               (2, Fraction(1, 5), Fraction(99, 100))])
+def test_selection_vs_exact_rational_brute_force(seed, alpha, c_min):
+    rng = np.random.default_rng(seed)
+    V, d, F_fixed = 40, 16, 900
+    tokens = (rng.zipf(1.3, size=500) % V).astype(np.int32)
+    f, order, C, R, U = exact_curves(tokens.tolist(), V, d, F_fixed, alpha)
+    res = so.select(tokens, V, d, float(F_fixed), float(alpha), float(c_min), 3, 35, fast_counts=False)
+    assert res["f"].tolist() == f and res["order"].tolist() == order
+    assert np.allclose(res["C"], [float(c) for c in C], rtol=0, atol=1e-15)
+    assert np.allclose(res["R"], [float(r) for r in R], rtol=0, atol=1e-15)
+    assert np.allclose(res["U"], [float(u) for u in U], rtol=0, atol=1e-15)
+    pen = [U[k - 1] if C[k - 1] >= c_min else Fraction(-1) for k in range(3, 36)]
+    best = max(pen)
+    assert res["k_star"] == 3 + pen.index(best)                        # smallest k among equal maxima
+    assert np.array_equal(so.frequencies(tokens, V), so.frequencies_fast(tokens, V))
+
+
+def test_limiting_cases_of_the_objective():
+    V, d, F = 1000, 64, 5e4
+    tokens = inputs.zipf_token_stream(V, 1.1, 20000, seed=5)
+    # alpha = 1: only coverage counts, the largest allowed vocabulary wins (first k reaching the final coverage)
+    r1 = so.select(tokens, V, d, F, 1.0, 0.0, 10, 900)
+    assert r1["C"][r1["k_star"] - 1] == r1["C"][899] and (r1["k_star"] == 10 or r1["C"][r1["k_star"] - 2] < r1["C"][899])
+    # alpha = 0: only the FLOPs proxy counts, the smallest feasible vocabulary wins
+    r0 = so.select(tokens, V, d, F, 0.0, 0.9, 10, 900)
+    assert r0["C"][r0["k_star"] - 1] >= 0.9 and r0["C"][r0["k_star"] - 2] < 0.9
+    # an unreachable coverage floor: every k is penalised to -1 and the first one is returned
+    rp = so.select(tokens, V, d, F, 0.5, 2.0, 10, 900)
+    assert rp["U_star"] == -1.0 and rp["k_star"] == 10
+    # coverage is a non-decreasing curve ending at 1 (Eq. 2)
+    assert np.all(np.diff(r1["C"]) >= 0) and r1["C"][-1] == 1.0
+    # a flat stream: every id equally frequent -> C(k) = k / V exactly and ids stay in id order
+    flat = np.repeat(np.arange(50, dtype=np.int32), 4)
+    rf = so.select(flat, 50, d, F, 0.5, 0.0, 1, 50)
+    assert rf["order"].tolist() == list(range(50)) and np.allclose(rf["C"], np.arange(1, 51) / 50.0, atol=1e-15)
