@@ -235,6 +235,14 @@ def run_ours(args):
     for _ in range(10):
         covered, frac = vt.vt_coverage(tok_dev, keep, V, cov_ws)
     coverage_us = (time.perf_counter() - t0) * 1e5
+    # the paper's selection step (Eq. 1-5 as an exhaustive scan) on the same stream, Table 1 constants
+    F_fixed = 2.0 * (3 * d) * d + 436.2e6 + 50.3e6
+    sel_ws = torch.empty(vt.vt_select_workspace_bytes(V), dtype=torch.uint8, device="cuda")
+    sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
+    t0 = time.perf_counter()
+    for _ in range(5):
+        sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
+    select_us = (time.perf_counter() - t0) * 2e5
 
     free, _ = torch.cuda.mem_get_info()
     nc = n_copies_for_cold(W_trim.numel() * 2, l2, free)
@@ -293,7 +301,10 @@ def run_ours(args):
         "once_per_model": {"compact_us": round(compact_us, 2),
                            "compact_GBs": round(2 * W_trim.numel() * 2 / compact_us / 1e3, 1),
                            "coverage_us_incl_sync": round(coverage_us, 2), "coverage_tokens": int(tokens.size),
-                           "coverage": frac},
+                           "coverage": frac,
+                           "select_vocab_us_incl_sync": round(select_us, 1),
+                           "select_vocab": {"alpha": 0.5, "c_min": 0.9, "k_range": [1000, 64000], "k_star": sel["k_star"],
+                                            "C": round(sel["C"], 6), "R": round(sel["R"], 6), "U": round(sel["U"], 6)}},
     }
 
     if rank == 0 and world == 1:

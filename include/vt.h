@@ -162,6 +162,34 @@ vt_status vt_coverage(const int32_t* token_ids, int64_t N,
                       uint64_t* covered_out, double* fraction_out,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Vocabulary-size selection (the paper's method, Sections 2.1-2.5), as an exhaustive scan over k:
+ *
+ *   f(v)  = occurrences of id v in token_ids (the stream is taken as already restricted to assistant
+ *           tokens, Section 2.2); ids outside [0, V_full) are ignored
+ *   order = ids by (f descending, id ascending)                     top-k most frequent, Section 2.1
+ *   C(k)  = (sum of the k largest f) / (sum of all f)               Eq. 2
+ *   R(k)  = 1 - (F_fixed + 2 d k) / (F_fixed + 2 d V_full)          Eq. 3
+ *   U(k)  = alpha C(k) + (1 - alpha) R(k);  U~(k) = U(k) if C(k) >= c_min, else -1       Eq. 4, 5
+ *   k*    = argmax of U~(k) over k_min <= k <= k_max, the smallest k among equal maxima   Eq. 1
+ *
+ * The paper searches k with 100 trials of a TPE optimiser; every k is evaluated here, which gives the exact
+ * optimum of the same objective.  All arithmetic is IEEE double without fused multiply-add.
+ *
+ *   token_ids  dev [N] int32            ranked_ids dev [V_full] int32 (out): ranked_ids[:k*] is the draft
+ *                                       vocabulary, i.e. keep_ids / d2t for the calls above
+ *   cum_counts dev [V_full] uint64 (out) or NULL: cum_counts[k-1] = occurrences covered by the top k
+ *   k_star     host (out);  C_star, R_star, U_star  host (out), each may be NULL
+ *   workspace  dev, 256-byte aligned, vt_select_workspace_bytes(V_full); contents are overwritten
+ * 1 <= k_min <= k_max <= V_full, 0 <= alpha <= 1, F_fixed >= 0, d >= 1.  SYNCHRONISES the stream.
+ * VT_ERR_EMPTY if N == 0 or no id falls inside [0, V_full). */
+size_t    vt_select_workspace_bytes(int V_full);
+vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed,
+                          double alpha, double c_min, int k_min, int k_max,
+                          int32_t* ranked_ids, uint64_t* cum_counts,
+                          int* k_star, double* C_star, double* R_star, double* U_star,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* vt_coverage for callers that must not allocate device memory.  (The paper has no counterpart: this
  * entry point exists for integration, not for the method.)
  *

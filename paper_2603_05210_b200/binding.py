@@ -37,6 +37,9 @@ SYMBOLS = {
     "vt_draft_head_host": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _sz, _p]),
     "vt_last_status": (_i, [_p, _p]),
     "vt_coverage": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p, _sz, _p]),
+    "vt_select_workspace_bytes": (_sz, [_i]),
+    "vt_select_vocab": (_i, [_p, _i64, _i, _i, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i, _i, _p, _p, _p, _p, _p,
+                            _p, _p, _sz, _p]),
     "vt_coverage_static": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p]),
     "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
@@ -197,6 +200,31 @@ def vt_coverage(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int,
                              ctypes.addressof(covered), ctypes.addressof(frac),
                              workspace.data_ptr(), workspace.numel(), _stream()), "vt_coverage")
     return int(covered.value), float(frac.value)
+
+
+def vt_select_workspace_bytes(V_full: int) -> int:
+    return int(lib().vt_select_workspace_bytes(V_full))
+
+
+def vt_select_vocab(token_ids: torch.Tensor, V_full: int, d: int, F_fixed: float, alpha: float, c_min: float,
+                    k_min: int, k_max: int, *, want_cum: bool = False, workspace: torch.Tensor | None = None) -> dict:
+    """k* and the frequency ranking (Eq. 1-5).  Returns k_star, C, R, U (at k*), ranked_ids [V_full] and, if asked, cum_counts."""
+    token_ids = _i32(token_ids, "token_ids")
+    dev = token_ids.device
+    ranked = torch.empty(V_full, dtype=torch.int32, device=dev)
+    cum = torch.empty(V_full, dtype=torch.int64, device=dev) if want_cum else None
+    if workspace is None:
+        workspace = torch.empty(vt_select_workspace_bytes(V_full), dtype=torch.uint8, device=dev)
+    k_star = ctypes.c_int(0)
+    C, R, U = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_double(0)
+    _check(lib().vt_select_vocab(token_ids.data_ptr() if token_ids.numel() else None, token_ids.numel(), V_full, d,
+                                 float(F_fixed), float(alpha), float(c_min), k_min, k_max, ranked.data_ptr(), _ptr(cum),
+                                 ctypes.addressof(k_star), ctypes.addressof(C), ctypes.addressof(R), ctypes.addressof(U),
+                                 workspace.data_ptr(), workspace.numel(), _stream()), "vt_select_vocab")
+    out = {"k_star": int(k_star.value), "C": float(C.value), "R": float(R.value), "U": float(U.value), "ranked_ids": ranked}
+    if want_cum:
+        out["cum_counts"] = cum
+    return out
 
 
 def vt_coverage_static(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int) -> tuple[int, float]:

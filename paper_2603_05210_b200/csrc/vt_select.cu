@@ -1,0 +1,274 @@
+// Vocabulary-size selection on the GPU: the paper's Method section as an exhaustive scan.
+//
+//   f(v)   token frequencies of the stream                               (Section 2.2)
+//   order  ids by (f descending, id ascending)                           (Section 2.1: top-k most frequent)
+//   C(k)   = sum of the k largest f / sum of all f                       (Eq. 2)
+//   R(k)   = 1 - (F_fixed + 2 d k) / (F_fixed + 2 d V)                   (Eq. 3)
+//   U(k)   = alpha C(k) + (1 - alpha) R(k),  U~(k) = U(k) if C(k) >= c_min else -1      (Eq. 4, 5)
+//   k*     = argmax over k in [k_min, k_max] of U~(k), smallest k among equal maxima    (Eq. 1)
+//
+// The paper samples 100 values of k with a TPE optimiser; evaluating every k costs one pass over a
+// 128K-entry prefix sum, so the scan returns the exact optimum of the same objective.  Three kernels:
+// a histogram with warp-aggregated atomics (HBM-bound read of the stream), a stable least-significant-
+// digit radix sort of (count, id) in one CTA (the vocabulary is only ~128K entries), and a scan +
+// objective + arg-max kernel in one CTA.  Doubles are combined with explicit round-to-nearest
+// operations so that no fused multiply-add changes a result against the fp64 definition.
+#include "vt_launch.h"
+
+namespace vt {
+
+struct SelectResult {
+    int k_star;
+    int pad;
+    double C, R, U;
+    unsigned long long total;
+    unsigned long long pad2[27];
+};
+static_assert(sizeof(SelectResult) == 256, "one line");
+
+// ------------------------------------------------------------------------------------------ histogram
+__global__ void __launch_bounds__(512) select_hist_kernel(const int32_t* __restrict__ token_ids, long long N, int V,
+                                                           unsigned int* __restrict__ counts) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += stride) {
+        const int t = token_ids[i];
+        const bool ok = (unsigned int)t < (unsigned int)V;
+        // lanes that hold the same id add once: a Zipf stream repeats its head tokens within a warp
+        const unsigned int active = __ballot_sync(__activemask(), ok);
+        if (ok) {
+            const unsigned int peers = __match_any_sync(active, t);
+            if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&counts[t], (unsigned int)__popc(peers));
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ sort
+// Stable LSD radix sort of V (key, id) pairs by one CTA of 1024 threads, 8 bits per pass.
+// key = key_max - count, so ascending keys are descending counts; ids start ascending and every pass is
+// stable, so equal counts stay in ascending id order.
+constexpr int kSortThreads = 1024;
+
+__global__ void __launch_bounds__(kSortThreads) select_sort_kernel(const unsigned int* __restrict__ counts, int V,
+                                                                    unsigned int key_max, int passes,
+                                                                    unsigned int* keyA, int* valA,
+                                                                    unsigned int* keyB, int* valB) {
+    __shared__ unsigned int base[256];                 // running output position of each digit
+    __shared__ unsigned int warp_cnt[32][256];         // per chunk: occurrences of each digit in each warp
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < V; i += kSortThreads) {
+        keyA[i] = key_max - counts[i];
+        valA[i] = i;
+    }
+    __syncthreads();
+    unsigned int* kin = keyA;
+    unsigned int* kout = keyB;
+    int* vin = valA;
+    int* vout = valB;
+    for (int pass = 0; pass < passes; ++pass) {
+        const int shift = 8 * pass;
+        if (tid < 256) base[tid] = 0;
+        __syncthreads();
+        for (int i = tid; i < V; i += kSortThreads) atomicAdd(&base[(kin[i] >> shift) & 255u], 1u);
+        __syncthreads();
+        if (warp == 0) {                                // exclusive scan of the 256 digit counts
+            unsigned int run = 0;
+            for (int c = 0; c < 8; ++c) {
+                const unsigned int v = base[c * 32 + lane];
+                unsigned int inc = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                base[c * 32 + lane] = run + inc - v;
+                run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+            }
+        }
+        __syncthreads();
+        for (int c0 = 0; c0 < V; c0 += kSortThreads) {
+            const int i = c0 + tid;
+            const bool ok = i < V;
+            const unsigned int key = ok ? kin[i] : 0u;
+            const int val = ok ? vin[i] : 0;
+            const unsigned int dg = ok ? (key >> shift) & 255u : 256u;     // 256: a lane past the end
+            for (int j = lane; j < 256; j += 32) warp_cnt[warp][j] = 0;
+            __syncwarp();
+            const unsigned int peers = __match_any_sync(0xFFFFFFFFu, dg);
+            const unsigned int before = __popc(peers & ((1u << lane) - 1u));
+            if (ok && before == 0) warp_cnt[warp][dg] = __popc(peers);
+            __syncthreads();
+            if (tid < 256) {                            // digit tid: warps in order, then advance its base
+                unsigned int run = base[tid];
+                for (int w = 0; w < 32; ++w) {
+                    const unsigned int n = warp_cnt[w][tid];
+                    warp_cnt[w][tid] = run;
+                    run += n;
+                }
+                base[tid] = run;
+            }
+            __syncthreads();
+            if (ok) {
+                const unsigned int pos = warp_cnt[warp][dg] + before;
+                kout[pos] = key;
+                vout[pos] = val;
+            }
+            __syncthreads();
+        }
+        unsigned int* tk = kin; kin = kout; kout = tk;
+        int* tv = vin; vin = vout; vout = tv;
+    }
+    // an odd number of passes leaves the result in the B buffers: bring it back to A
+    if (kin != keyA) {
+        for (int i = tid; i < V; i += kSortThreads) {
+            keyA[i] = kin[i];
+            valA[i] = vin[i];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ scan + objective
+__global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* __restrict__ key_sorted,
+                                                           const int* __restrict__ val_sorted, int V,
+                                                           unsigned int key_max, int d, double F_fixed, double alpha,
+                                                           double c_min, int k_min, int k_max,
+                                                           unsigned long long* __restrict__ cum,
+                                                           int32_t* __restrict__ ranked_ids,
+                                                           unsigned long long* __restrict__ cum_out,
+                                                           SelectResult* result) {
+    __shared__ unsigned long long warp_tot[32];
+    __shared__ unsigned long long carry_s;
+    __shared__ double best_u[32];
+    __shared__ int best_k[32];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) carry_s = 0ull;
+    __syncthreads();
+    for (int c0 = 0; c0 < V; c0 += 1024) {              // inclusive prefix sum of the sorted counts
+        const int i = c0 + tid;
+        unsigned long long v = i < V ? (unsigned long long)(key_max - key_sorted[i]) : 0ull;
+        if (i < V) ranked_ids[i] = val_sorted[i];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long n = __shfl_up_sync(0xFFFFFFFFu, v, o);
+            if (lane >= o) v += n;
+        }
+        if (lane == 31) warp_tot[warp] = v;
+        __syncthreads();
+        unsigned long long off = carry_s;
+        for (int w = 0; w < warp; ++w) off += warp_tot[w];
+        v += off;
+        if (i < V) {
+            cum[i] = v;
+            if (cum_out) cum_out[i] = v;
+        }
+        __syncthreads();
+        if (tid == 1023) carry_s = v;
+        __syncthreads();
+    }
+    const unsigned long long total = carry_s;
+    const double tot_d = (double)total;
+    const double two_d = __dmul_rn(2.0, (double)d);
+    const double denom = __dadd_rn(F_fixed, __dmul_rn(two_d, (double)V));
+    const double one_minus_alpha = __dsub_rn(1.0, alpha);
+    double bu = -2.0, bc = 0.0, br = 0.0;
+    int bk = 0x7FFFFFFF;
+    if (total > 0) {
+        for (int k = k_min + tid; k <= k_max; k += 1024) {    // each thread meets its k in ascending order
+            const double C = __ddiv_rn((double)cum[k - 1], tot_d);
+            const double R = __dsub_rn(1.0, __ddiv_rn(__dadd_rn(F_fixed, __dmul_rn(two_d, (double)k)), denom));
+            const double U = __dadd_rn(__dmul_rn(alpha, C), __dmul_rn(one_minus_alpha, R));
+            const double Up = C >= c_min ? U : -1.0;
+            if (Up > bu) { bu = Up; bk = k; bc = C; br = R; }
+        }
+    }
+    // arg-max over the block: larger value wins, equal values go to the smaller k
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ou = __shfl_xor_sync(0xFFFFFFFFu, bu, o);
+        const int ok = __shfl_xor_sync(0xFFFFFFFFu, bk, o);
+        const double oc = __shfl_xor_sync(0xFFFFFFFFu, bc, o);
+        const double orr = __shfl_xor_sync(0xFFFFFFFFu, br, o);
+        if (ou > bu || (ou == bu && ok < bk)) { bu = ou; bk = ok; bc = oc; br = orr; }
+    }
+    __shared__ double best_c[32], best_r[32];
+    if (lane == 0) { best_u[warp] = bu; best_k[warp] = bk; best_c[warp] = bc; best_r[warp] = br; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 32; ++w)
+            if (best_u[w] > bu || (best_u[w] == bu && best_k[w] < bk)) { bu = best_u[w]; bk = best_k[w]; bc = best_c[w]; br = best_r[w]; }
+        result->k_star = total > 0 ? bk : 0;
+        result->C = bc;
+        result->R = br;
+        result->U = bu;
+        result->total = total;
+    }
+}
+
+static inline size_t up256s(size_t b) { return (b + 255) & ~(size_t)255; }
+
+}  // namespace vt
+
+using namespace vt;
+
+extern "C" size_t vt_select_workspace_bytes(int V_full) {
+    if (V_full < 1) return 0;
+    const size_t v = (size_t)V_full;
+    return 256 + up256s(v * 4) * 5 + up256s(v * 8);     // result | counts | keyA keyB valA valB | cum
+}
+
+extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed, double alpha,
+                                     double c_min, int k_min, int k_max, int32_t* ranked_ids, uint64_t* cum_counts,
+                                     int* k_star, double* C_star, double* R_star, double* U_star, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (!ranked_ids || !k_star || (!token_ids && N > 0)) return VT_ERR_NULL;
+    if (V_full < 1 || d < 1 || N < 0 || k_min < 1 || k_max < k_min || k_max > V_full || !(alpha >= 0.0 && alpha <= 1.0) ||
+        !(F_fixed >= 0.0))
+        return VT_ERR_SHAPE;
+    if (N == 0) return VT_ERR_EMPTY;
+    if ((reinterpret_cast<uintptr_t>(token_ids) & 3) || (reinterpret_cast<uintptr_t>(ranked_ids) & 3) ||
+        (cum_counts && (reinterpret_cast<uintptr_t>(cum_counts) & 7)))
+        return VT_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < vt_select_workspace_bytes(V_full))
+        return VT_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char* base = reinterpret_cast<unsigned char*>(workspace);
+    const size_t a4 = up256s((size_t)V_full * 4);
+    SelectResult* result = reinterpret_cast<SelectResult*>(base);
+    unsigned int* counts = reinterpret_cast<unsigned int*>(base + 256);
+    unsigned int* keyA = reinterpret_cast<unsigned int*>(base + 256 + a4);
+    unsigned int* keyB = reinterpret_cast<unsigned int*>(base + 256 + 2 * a4);
+    int* valA = reinterpret_cast<int*>(base + 256 + 3 * a4);
+    int* valB = reinterpret_cast<int*>(base + 256 + 4 * a4);
+    unsigned long long* cum = reinterpret_cast<unsigned long long*>(base + 256 + 5 * a4);
+
+    cudaError_t e = cudaMemsetAsync(base, 0, 256 + a4, st);          // result and counts
+    if (e != cudaSuccess) return cuda_fail(e);
+    int sms = 0;
+    vt_status r = device_sm_count(&sms);
+    if (r != VT_OK) return r;
+    const int grid = (int)std::max<long long>(1, std::min<long long>((N + 511) / 512, (long long)sms * 4));
+    select_hist_kernel<<<grid, 512, 0, st>>>(token_ids, N, V_full, counts);
+    count_launch();
+    // a count is at most N: sort only the bits that can be set
+    int bits = 1;
+    while (bits < 32 && (1ll << bits) <= N) ++bits;
+    const unsigned int key_max = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
+    const int passes = (bits + 7) / 8;
+    select_sort_kernel<<<1, kSortThreads, 0, st>>>(counts, V_full, key_max, passes, keyA, valA, keyB, valB);
+    count_launch();
+    select_scan_kernel<<<1, 1024, 0, st>>>(keyA, valA, V_full, key_max, d, F_fixed, alpha, c_min, k_min, k_max, cum,
+                                           ranked_ids, reinterpret_cast<unsigned long long*>(cum_counts), result);
+    count_launch();
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    SelectResult host;
+    e = cudaMemcpyAsync(&host, result, sizeof host, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (host.total == 0) return VT_ERR_EMPTY;                       // no token id fell inside [0, V_full)
+    *k_star = host.k_star;
+    if (C_star) *C_star = host.C;
+    if (R_star) *R_star = host.R;
+    if (U_star) *U_star = host.U;
+    return VT_OK;
+}
