@@ -29,7 +29,9 @@ def build(force: bool = False) -> str:
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
+        # VT_ORACLE_LIB points the loader at another build of the same source: the mutation test uses it to
+        # check that the pins notice a planted mistake
+        lib = ctypes.CDLL(os.environ.get("VT_ORACLE_LIB") or build())
         lib.vto_bf16_to_f64.restype = ctypes.c_double
         lib.vto_bf16_to_f64.argtypes = [ctypes.c_uint16]
         lib.vto_num_threads.restype = ctypes.c_int

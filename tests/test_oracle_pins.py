@@ -158,6 +158,10 @@ def test_log_softmax_closed_forms(oracle):
         lp, _ = oracle.log_softmax(np.array([[delta, 0.0]]))
         assert abs(lp[0, 0] + math.log1p(math.exp(-delta))) < 1e-14
         assert abs(lp[0, 1] + delta + math.log1p(math.exp(-delta))) < 1e-13
+    # a spread far beyond exp's range: only the row maximum may be factored out
+    lp, lse = oracle.log_softmax(np.array([[1000.0, 0.0, -1000.0], [-2000.0, -900.0, -901.0]]))
+    assert np.all(np.isfinite(lse)) and lse[0] == 1000.0 and lp[0, 0] == 0.0 and lp[0, 2] == -2000.0
+    assert abs(lse[1] - (-900.0 + math.log1p(math.exp(-1.0)))) < 1e-12
     # three classes, hand value: log(1 + 2 + 4) with logits log 1, log 2, log 4
     lp, lse = oracle.log_softmax(np.log(np.array([[1.0, 2.0, 4.0]])))
     assert abs(lse[0] - math.log(7.0)) < 1e-14
