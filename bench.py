@@ -46,7 +46,7 @@ def head_bytes(d, Vt, M, k):
 # DRAM traffic of one head launch on the bench workload from the ncu capture summarised in
 # profiles/head_mma_d4096_vt32000_m8.md (dram__bytes_read.sum + dram__bytes_write.sum), valid while the
 # kernel sources still hash to the value recorded there.
-NCU_TRAFFIC = {"bytes": 262_353_152 + 3_809_280, "source_hash": "5f3476797b48d090",
+NCU_TRAFFIC = {"bytes": 271_346_688 + 3_662_848, "source_hash": "9050caa4aa8c15a1",
                "sources": ("paper_2603_05210_b200/csrc/vt_head_mma.cu", "paper_2603_05210_b200/csrc/vt_common.cuh")}
 
 
