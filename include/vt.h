@@ -230,6 +230,15 @@ vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V
 vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
                    int32_t* target_ids, void* stream);
 
+/* The index buffers an EAGLE-3 style draft stores with its weights (Section 1: "draft-to-target and
+ * target-to-draft index buffers"), derived from keep_ids:
+ *   d2t_offsets[i] = keep_ids[i] - i        (target id = draft index + offset), dev [V_trim] int32 or NULL
+ *   t2d_mask[v]    = 1 if v is kept else 0,                                      dev [V_full] uint8 or NULL
+ * At least one output must be given.  The head calls above take absolute ids (keep_ids itself as d2t); this
+ * call only converts for checkpoints that use the offset form.  Asynchronous. */
+vt_status vt_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full,
+                        int32_t* d2t_offsets, uint8_t* t2d_mask, void* stream);
+
 /* Number of kernels the last call of this thread launched (for launch accounting). */
 int vt_last_launch_count(void);
 

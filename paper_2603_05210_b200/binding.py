@@ -43,6 +43,7 @@ SYMBOLS = {
     "vt_coverage_static": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p]),
     "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
+    "vt_vocab_maps": (_i, [_p, _i, _i, _p, _p, _p]),
     "vt_last_launch_count": (_i, []),
 }
 
@@ -260,6 +261,16 @@ def vt_remap(draft_ids: torch.Tensor, d2t: torch.Tensor) -> torch.Tensor:
     _check(lib().vt_remap(draft_ids.data_ptr(), d2t.data_ptr(), draft_ids.numel(), d2t.numel(), out.data_ptr(),
                           _stream()), "vt_remap")
     return out
+
+
+def vt_vocab_maps(keep_ids: torch.Tensor, V_full: int) -> tuple[torch.Tensor, torch.Tensor]:
+    """(d2t offsets [V_trim] int32, t2d membership mask [V_full] uint8) in the form EAGLE-3 checkpoints store."""
+    keep_ids = _i32(keep_ids, "keep_ids")
+    off = torch.empty_like(keep_ids)
+    mask = torch.empty(V_full, dtype=torch.uint8, device=keep_ids.device)
+    _check(lib().vt_vocab_maps(keep_ids.data_ptr(), keep_ids.numel(), V_full, off.data_ptr(), mask.data_ptr(), _stream()),
+           "vt_vocab_maps")
+    return off, mask
 
 
 def vt_last_launch_count() -> int:

@@ -310,4 +310,13 @@ vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int 
     return launch_remap(draft_ids, d2t, n, V_trim, target_ids, (cudaStream_t)stream);
 }
 
+vt_status vt_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full, int32_t* d2t_offsets, uint8_t* t2d_mask,
+                        void* stream) {
+    g_launches = 0;
+    if (!keep_ids || (!d2t_offsets && !t2d_mask)) return VT_ERR_NULL;
+    if (V_full < 1 || V_trim < 1 || V_trim > V_full) return VT_ERR_SHAPE;
+    if (!aligned(keep_ids, 4) || (d2t_offsets && !aligned(d2t_offsets, 4))) return VT_ERR_ALIGN;
+    return launch_vocab_maps(keep_ids, V_trim, V_full, d2t_offsets, t2d_mask, (cudaStream_t)stream);
+}
+
 }  // extern "C"

@@ -76,6 +76,33 @@ vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, 
 }
 
 // ------------------------------------------------------------------------------------------
+// The two index buffers an EAGLE-3 style draft carries: draft-to-target as offsets
+// (target id = draft index + offset) and target-to-draft as a membership flag per target id.
+// ------------------------------------------------------------------------------------------
+__global__ void vocab_maps_kernel(const int32_t* __restrict__ keep_ids, int V_trim, int V_full,
+                                  int32_t* __restrict__ d2t_offsets, unsigned char* __restrict__ t2d_mask) {
+    const int stride = gridDim.x * blockDim.x;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < V_trim; i += stride) {
+        const int v = keep_ids[i];
+        if (d2t_offsets) d2t_offsets[i] = v - i;
+        if (t2d_mask && v >= 0 && v < V_full) t2d_mask[v] = 1;
+    }
+}
+
+vt_status launch_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full, int32_t* d2t_offsets,
+                            unsigned char* t2d_mask, cudaStream_t st) {
+    if (t2d_mask) {
+        cudaError_t e = cudaMemsetAsync(t2d_mask, 0, (size_t)V_full, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    const int grid = std::max(1, std::min((V_trim + 255) / 256, 592));
+    vocab_maps_kernel<<<grid, 256, 0, st>>>(keep_ids, V_trim, V_full, d2t_offsets, t2d_mask);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
 // Membership bitmap of the kept set (bit v of the bitmap = "v is in V_d"); the same pass counts
 // out-of-range ids and ids seen twice.
 // ------------------------------------------------------------------------------------------

@@ -203,6 +203,10 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
     int* last_flag = const_cast<int*>(abort_flag) + 1;
 
     const int n_epi_warps = (p.m_count + 31) / 32;
+    if (warp == 4 && lane == 0) {      // descriptor fetches overlap the barrier set-up below
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
+    }
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8u * s, 1);

@@ -38,6 +38,8 @@ vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st);
 
 vt_status launch_compact(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim,
                          void* W_trim, cudaStream_t st);
+vt_status launch_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full, int32_t* d2t_offsets,
+                            unsigned char* t2d_mask, cudaStream_t st);
 vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
                        int32_t* target_ids, cudaStream_t st);
 

@@ -92,6 +92,18 @@ def test_remap_bit_exact(vt, oracle):
     assert got[0, 0] == -1 and got[1, 1] == -1 and np.array_equal(got[2:], oracle.remap(idx, d2t)[2:])
 
 
+def test_vocab_maps_bit_exact(vt):
+    rng = np.random.default_rng(4)
+    V, Vt = 128256, 13264
+    keep = rng.permutation(V)[:Vt].astype(np.int32)
+    off, mask = vt.vt_vocab_maps(dev_i32(keep), V)
+    assert np.array_equal(off.cpu().numpy(), keep - np.arange(Vt, dtype=np.int32))      # target = draft index + offset
+    want = np.zeros(V, dtype=np.uint8)
+    want[keep] = 1
+    assert np.array_equal(mask.cpu().numpy(), want)
+    assert int(mask.sum()) == Vt
+
+
 # ------------------------------------------------------------------------------ logits
 LOGIT_SHAPES = [(1, 8, 1), (1, 64, 7), (3, 64, 127), (8, 2048, 129), (2, 3072, 1000), (4, 4096, 4380),
                 (9, 2048, 300), (17, 64, 1025), (3, 5120, 700), (5, 200, 2000), (64, 512, 333), (1, 8192, 150)]
