@@ -110,6 +110,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return true;
 }
 
+// Programmatic dependent launch.  A head kernel is launched with the programmatic-serialization attribute:
+// its CTAs may become resident while the previous kernel in the stream is still finishing (for back-to-back
+// head calls: while the last CTA of the previous call merges), run their set-up that touches no global
+// memory, and then wait here until that previous kernel has completed and its writes are visible.  Without
+// the attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.
 // Both addresses and the size must be multiples of 16 bytes.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

@@ -101,6 +101,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         fence_mbar_init();
     }
     for (int i = tid; i < kGemvConsumers * NV * KS; i += blockDim.x) lists[i] = 0ull;
+    grid_dependency_wait();            // nothing above touched global memory
+    if (tid == 0) grid_launch_dependents();
     {   // hidden states of this pass; pad rows (m >= m_count) repeat the last real row and are never read out
         const int nchunks = d >> 3;
         for (int i = tid; i < MP * nchunks; i += blockDim.x) {
@@ -244,9 +246,9 @@ static vt_status launch_one(const GemvParams& p, int grid, cudaStream_t st) {
         if (e != cudaSuccess) return cuda_fail(e);
         configured_device = dev;
     }
-    kern<<<grid, kGemvThreads, p.total_smem, st>>>(p);
+    cudaError_t e = launch_pdl(kern, grid, kGemvThreads, p.total_smem, st, p);
     count_launch();
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
 }
 

@@ -242,6 +242,9 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                      ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // everything above touched only shared memory, tensor memory and kernel parameters
+    grid_dependency_wait();
+    if (tid == 0) grid_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -601,9 +604,9 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.bar_off = (uint32_t)((p.list_off + list_bytes + 127) & ~(size_t)127);
         p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
 
-        head_mma_kernel<<<grid, kMmaThreads, p.total_smem, st>>>(tmW, tmWt, tmH, p);
+        cudaError_t e = launch_pdl(head_mma_kernel, grid, kMmaThreads, p.total_smem, st, tmW, tmWt, tmH, p);
         count_launch();
-        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return VT_OK;

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <utility>
 
 #include "vt_common.cuh"
 
@@ -29,6 +30,22 @@ vt_status device_sm_count(int* sms);
 inline int head_grid(int sms, int Vt, int min_rows_per_cta = 1) {
     const int by_rows = (Vt + min_rows_per_cta - 1) / min_rows_per_cta;
     return std::max(1, std::min(std::min(sms, kMaxParts), by_rows));
+}
+
+// Launches with programmatic stream serialization (see grid_dependency_wait in vt_common.cuh).
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 bool gemv_supports(int d);

@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const HeadOut o, i
         mbar_init(smem_u32(&bar), 1);
         fence_mbar_init();
     }
+    grid_dependency_wait();            // the head kernel's records must be complete
     __syncthreads();
     const int m_begin = blockIdx.x * kMergeRowsPerCta;
     const int m_count = min(kMergeRowsPerCta, o.M - m_begin);
@@ -39,9 +40,9 @@ vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st) {
         configured_device = dev;
     }
     const int grid = (o.M + kMergeRowsPerCta - 1) / kMergeRowsPerCta;
-    merge_kernel<<<grid, kMergeThreads, want, st>>>(o, P, (uint32_t)want);
+    cudaError_t e = launch_pdl(merge_kernel, grid, kMergeThreads, want, st, o, P, (uint32_t)want);
     count_launch();
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
 }
 
