@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
-    const int Vt = p.out.Vt, d = p.d, k = p.out.k, M = p.out.M;
+    const int Vt = p.out.Vt, d = p.d, k = p.out.k;
     const int row_begin = (int)((long long)cta * Vt / G);
     const int row_end = (int)((long long)(cta + 1) * Vt / G);
     const int nrows = row_end - row_begin;

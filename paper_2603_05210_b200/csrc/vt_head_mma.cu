@@ -31,13 +31,7 @@ struct MmaParams {
     HeadOut out;
     int m_begin, m_count;     // draft rows of this pass
     int d;
-    int NT;                   // vocabulary rows per main tile (multiple of 16, <= 256)
-    int n_main;               // main tiles a CTA with the most rows has
-    int NT_tail;              // rows of the short tile that follows them (0: none); its epilogue is the only one
-                              // that cannot hide behind the weight stream, so it is kept short
-    uint32_t idesc_tail;
-    int kb_tail;              // k-blocks per stage and bytes per k-block while the tail tile streams
-    uint32_t blk_tail;
+    int NT;                   // vocabulary rows per tile (multiple of 16, <= 256)
     int nk;                   // 64-column k-blocks per tile
     int kb_per_stage;         // k-blocks one ring stage holds (one barrier hand-over per stage)
     uint32_t blk_bytes;       // bytes of one k-block in a stage: (A slot +) B slot, multiple of 1024
@@ -173,8 +167,7 @@ __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, 
 // through shared memory so that a whole warp works on one draft row at a time (warp_topk_update), which
 // keeps all 32 lanes busy when there are only a few draft rows.
 __global__ void __launch_bounds__(kMmaThreads, 1)
-head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWt,
-                const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
+head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, const MmaParams p) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -182,15 +175,11 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
-    const int Vt = p.out.Vt, k = p.out.k, M = p.out.M, NT = p.NT, S = p.n_stages, nk = p.nk;
+    const int Vt = p.out.Vt, k = p.out.k, NT = p.NT, S = p.n_stages, nk = p.nk;
     const int row_begin = (int)((long long)cta * Vt / G);
     const int row_end = (int)((long long)(cta + 1) * Vt / G);
     const int nrows = row_end - row_begin;
-    // tiles of this CTA: up to n_main tiles of NT rows, then (if rows remain) one tile of NT_tail rows
-    const int main_here = min(p.n_main, (nrows + NT - 1) / NT);
-    const bool tail_here = p.NT_tail > 0 && nrows > p.n_main * NT;
-    const int ntiles = main_here + (tail_here ? 1 : 0);
-    auto tile_rows = [&](int t) { return (tail_here && t == ntiles - 1) ? p.NT_tail : NT; };
+    const int ntiles = (nrows + NT - 1) / NT;
 
     unsigned long long* epi = reinterpret_cast<unsigned long long*>(smem + p.list_off);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
@@ -272,11 +261,10 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * NT;
-                const bool is_tail = tail_here && t == ntiles - 1;
-                const CUtensorMap* mapW = is_tail ? &tmWt : &tmW;
-                const uint32_t b_tx = (uint32_t)tile_rows(t) * 128u;
-                const int kbs = is_tail ? p.kb_tail : p.kb_per_stage;
-                const uint32_t blk = is_tail ? p.blk_tail : p.blk_bytes;
+                const CUtensorMap* mapW = &tmW;
+                const uint32_t b_tx = p.b_tx;
+                const int kbs = p.kb_per_stage;
+                const uint32_t blk = p.blk_bytes;
                 for (int ks = 0; ks < nk; ks += kbs) {
                     if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
@@ -317,10 +305,9 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
-                const bool is_tail = tail_here && t == ntiles - 1;
-                const uint32_t idesc = is_tail ? p.idesc_tail : p.idesc;
-                const int kbs = is_tail ? p.kb_tail : p.kb_per_stage;
-                const uint32_t blk_units = (is_tail ? p.blk_tail : p.blk_bytes) >> 4;
+                const uint32_t idesc = p.idesc;
+                const int kbs = p.kb_per_stage;
+                const uint32_t blk_units = p.blk_bytes >> 4;
                 for (int ks = 0; ks < nk; ks += kbs) {
                     if (!mbar_wait(bar_full + 8u * s, phase)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
@@ -372,7 +359,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 tc_fence_after();
             }
             const int row0 = row_begin + t * NT;
-            const int ncols = min(tile_rows(t), row_end - row0);
+            const int ncols = min(NT, row_end - row0);
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kAccStride);
             for (int c0 = 0; c0 < ncols; c0 += 32) {
                 const int nv = min(32, ncols - c0);
@@ -486,33 +473,20 @@ static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, in
     return cr == CUDA_SUCCESS ? VT_OK : driver_fail((int)cr);
 }
 
-// Tiling of the most rows a CTA owns: n_main tiles of NT rows plus, optionally, one short tail tile whose
-// epilogue (the only one nothing streams behind) would be shorter.  Measured on B200 a 48- or 64-row tail
-// streams too slowly to pay for itself (an MMA costs 45 cycles however few rows it covers, and every ring
-// stage a barrier hand-over), so kMaxTailRows is 0 and the search only picks the main tile: the multiple
-// of 16 that covers the rows with the least padding - rows a tile loads past the CTA's range are wasted
-// HBM traffic - preferring heights just below 128 among equals (measured: 2 x 112 beats 1 x 224).
-struct Tiling { int NT, n_main, NT_tail; };
-constexpr int kMaxTailRows = 0;
-static Tiling choose_tiling(int rows) {
-    // tiles below 96 rows only when the CTA has fewer rows than that: every ring stage costs a barrier
-    // hand-over and every MMA 45 cycles however few rows it covers
-    if (rows <= 96) return Tiling{((rows + 15) / 16) * 16, 1, 0};
-    Tiling best{256, (rows + 255) / 256, 0};
-    int best_cost = 1 << 30;
+// Tile height for the most rows a CTA owns: a multiple of 16, at least 96 unless the CTA has fewer rows
+// (every ring stage costs a barrier hand-over and every MMA 45 cycles however few rows it covers), with the
+// least padding - rows a tile loads past the CTA's range are wasted HBM traffic - and, among equals, the
+// height nearest 128 from below: with two or more tiles per CTA all epilogues but the last hide behind the
+// stream, and the last one is short (measured: 2 x 112 beats 1 x 224; tiles of 48-64 rows stream too slowly).
+static int choose_tile_rows(int rows) {
+    if (rows <= 96) return ((rows + 15) / 16) * 16;
+    int best = 256, best_cost = 1 << 30;
     for (int nt = 96; nt <= 256; nt += 16) {
-        for (int tail = 0; tail <= kMaxTailRows; tail += 16) {
-            if (tail > 0 && (tail < 48 || tail >= rows)) continue;
-            const int n_main = (rows - tail + nt - 1) / nt;
-            if (tail > 0 && rows <= n_main * nt) continue;          // the tail would be empty
-            const int pad = n_main * nt + tail - rows;
-            // least padding first; among equals the height nearest 128 from below: two or more tiles per CTA let
-            // all but the last epilogue hide behind the stream, and the last one is half as long
-            const int cost = pad * 1024 + (tail > 0 ? tail : (nt <= 128 ? 128 - nt : nt));
-            if (cost < best_cost) {
-                best_cost = cost;
-                best = Tiling{nt, n_main, tail};
-            }
+        const int pad = (rows + nt - 1) / nt * nt - rows;
+        const int cost = pad * 1024 + (nt <= 128 ? 128 - nt : nt);
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = nt;
         }
     }
     return best;
@@ -525,8 +499,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
     const int rows_per_cta = (c.Vt + grid - 1) / grid;
-    const Tiling tiling = choose_tiling(rows_per_cta);
-    const int NT = tiling.NT;
+    const int NT = choose_tile_rows(rows_per_cta);
 
     static int configured_device = -1;
     int dev = 0;
@@ -540,11 +513,6 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     CUtensorMap tmW;
     r = make_map(&tmW, c.W, c.Vt, c.d, NT);
     if (r != VT_OK) return r;
-    CUtensorMap tmWt = tmW;
-    if (tiling.NT_tail > 0) {
-        r = make_map(&tmWt, c.W, c.Vt, c.d, tiling.NT_tail);
-        if (r != VT_OK) return r;
-    }
 
     for (int m0 = 0; m0 < c.M; m0 += 128) {
         const int mc = std::min(128, c.M - m0);
@@ -558,8 +526,6 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.m_count = mc;
         p.d = c.d;
         p.NT = NT;
-        p.n_main = tiling.n_main;
-        p.NT_tail = tiling.NT_tail;
         p.nk = (c.d + kBoxK - 1) / kBoxK;
         p.a_tx = (uint32_t)mc * 128u;
         p.b_tx = (uint32_t)NT * 128u;
@@ -572,11 +538,8 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.kb_per_stage = std::max(1, std::min(4, (int)((28 * 1024 + p.blk_bytes / 2) / p.blk_bytes)));
         p.kb_per_stage = std::min(p.kb_per_stage, p.nk);
         p.stage_bytes = p.blk_bytes * p.kb_per_stage;
-        p.blk_tail = (p.h_resident ? 0u : p.a_slot) + (((uint32_t)tiling.NT_tail * 128u + 1023u) & ~1023u);
-        p.kb_tail = tiling.NT_tail > 0 ? std::max(1, std::min(p.nk, (int)(p.stage_bytes / p.blk_tail))) : 1;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N = NT, M = 128
         p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        p.idesc_tail = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tiling.NT_tail >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         // epilogue scratch: lists, candidate staging and a transpose buffer per epilogue warp; the fewer draft
         // rows a warp has, the more columns it can afford to select from at a time
         const int epi_warps = (mc + 31) / 32;
@@ -604,7 +567,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.bar_off = (uint32_t)((p.list_off + list_bytes + 127) & ~(size_t)127);
         p.total_smem = (uint32_t)(p.bar_off + bar_bytes + 1024);
 
-        cudaError_t e = launch_pdl(head_mma_kernel, grid, kMmaThreads, p.total_smem, st, tmW, tmWt, tmH, p);
+        cudaError_t e = launch_pdl(head_mma_kernel, grid, kMmaThreads, p.total_smem, st, tmW, tmH, p);
         count_launch();
         if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e);
