@@ -19,7 +19,7 @@ VT_OK = 0
 VT_ERR_NULL, VT_ERR_SHAPE, VT_ERR_ALIGN, VT_ERR_RANGE, VT_ERR_DUP = 1, 2, 3, 4, 5
 VT_ERR_EMPTY, VT_ERR_WORKSPACE, VT_ERR_TIMEOUT, VT_ERR_CUDA, VT_ERR_UNSUPPORTED = 6, 7, 8, 9, 10
 VT_MAX_K = 64
-VT_PATH_AUTO, VT_PATH_GEMV, VT_PATH_MMA = 0, 1, 2
+VT_PATH_AUTO, VT_PATH_GEMV, VT_PATH_MMA, VT_PATH_MMA_SMALL = 0, 1, 2, 3
 
 # every symbol include/vt.h declares: name -> (restype, argtypes)
 _p, _i, _i64, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t

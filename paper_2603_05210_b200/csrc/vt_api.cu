@@ -70,7 +70,9 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
     return o;
 }
 
-// M at or below which the CUDA-core GEMV is used when both paths can run the shape.
+// M at or below which the vocabulary-rows-on-lanes tensor-core kernel is tried first (it needs h to fit in
+// shared memory), and M at or below which the CUDA-core GEMV comes next.
+constexpr int kAutoSmallMaxM = 16;
 constexpr int kAutoGemvMaxM = 2;
 
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
@@ -80,8 +82,12 @@ static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
         r = launch_head_gemv(c, st, &grid);
     } else if (path == VT_PATH_MMA) {
         r = launch_head_mma(c, st, &grid);
+    } else if (path == VT_PATH_MMA_SMALL) {
+        r = launch_head_mma_small(c, st, &grid);
     } else if (path != VT_PATH_AUTO) {
         return VT_ERR_SHAPE;
+    } else if (c.M <= kAutoSmallMaxM && (r = launch_head_mma_small(c, st, &grid)) != VT_ERR_UNSUPPORTED) {
+        // launched (or failed for a reason another path would not cure)
     } else if (c.M <= kAutoGemvMaxM && gemv_supports(c.d)) {
         r = launch_head_gemv(c, st, &grid);
     } else {

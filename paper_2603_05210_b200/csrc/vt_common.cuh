@@ -24,10 +24,13 @@ namespace vt {
 constexpr int kMaxParts = 256;             // upper bound on CTAs that contribute partials
 constexpr size_t kHeaderBytes = 256;
 
+constexpr int kRowTickets = 16;            // draft rows that can be merged row by row (one ticket each)
+
 struct WsHeader {
     unsigned int ticket;     // CTAs that have published their partials in the running call
     unsigned int status;     // bit 0: a bounded wait ran out
-    unsigned int pad[62];
+    unsigned int row_ticket[kRowTickets];   // per draft row: CTAs that have published that row (row-wise merge)
+    unsigned int pad[62 - kRowTickets];
 };
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header is one 256-byte line");
 
@@ -45,6 +48,16 @@ __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
 
 // Record of (CTA p, draft row m).
 #define VT_REC(o, p, m) ((o).recs + (size_t)(p) * ws_pitch((o).M, (o).k) + (size_t)(m) * ws_slots((o).k))
+
+// Row-major records (the row-wise merge of the few-draft-rows kernel): draft row m owns kMaxParts * (k + 1)
+// consecutive u64 of the same record area,
+//   heads [kMaxParts]          every CTA's best key        (one coalesced read finds the lists that matter)
+//   ms    [kMaxParts]          every CTA's (max, sum-exp)
+//   rest  [kMaxParts][k - 1]   every CTA's 2nd .. k-th key
+// M * kMaxParts * (k + 1) <= kMaxParts * ws_pitch(M, k), so the area vt_workspace_bytes sizes holds either layout.
+#define VT_ROW_HEADS(o, m) ((o).recs + (size_t)(m) * kMaxParts * ((o).k + 1))
+#define VT_ROW_MS(o, m) (VT_ROW_HEADS(o, m) + kMaxParts)
+#define VT_ROW_REST(o, m, p) (VT_ROW_HEADS(o, m) + 2 * kMaxParts + (size_t)(p) * ((o).k - 1))
 
 struct HeadOut {
     const int32_t* d2t;   // null: report draft indices as target ids
@@ -193,6 +206,74 @@ __device__ __forceinline__ unsigned long long warp_max_key(unsigned long long v)
     return ((unsigned long long)mhi << 32) | mlo;
 }
 
+// Top-k update of one draft row by a whole warp.  `vals` is the row's logits for `ncols` consecutive
+// vocabulary columns (first column = vocabulary row `col0`), in shared memory; `list` is the row's k best
+// so far (descending keys, 0 = empty) and `tau` the logit of its k-th best (-inf while the list is not
+// full).  Lane L looks at columns L, L+32, ...
+//   1. bound: the 32 lanes form 8, 16 or 32 groups (whichever is >= k; k <= 32); the smallest group maximum
+//      has at least k logits at or above it, so nothing below it can be among the k best of these columns;
+//   2. the logits above tau (strictly: a later row loses a tie) and not below the bound are the candidates;
+//      a ballot per column group gives each its slot in `cbuf`, and the current list follows them;
+//   3. every entry of cbuf counts the entries larger than itself - its rank - and the entries of rank < k
+//      form the new list.  Keys are distinct, so ranks are too.  No step depends on the previous candidate,
+//      unlike an insertion loop.
+// The same pass folds the columns into the row's running (max, sum-exp) in *ms.
+// Returns the new tau.  All lanes must call it; NI * 32 >= ncols; `cbuf` holds NI * 32 + k keys.
+template <int NI>
+__device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, int col0, unsigned long long* list,
+                                                  int k, float tau, unsigned long long* cbuf, float2* ms, int lane) {
+    float v[NI];
+    float lmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int c = lane + 32 * i;
+        v[i] = c < ncols ? vals[c] : -INFINITY;
+        lmax = fmaxf(lmax, v[i]);
+    }
+    {   // running log-sum-exp of the row: (max, sum of exp(x - max)), folded over these columns by the warp
+        const float2 old = *ms;
+        const float bmax = warp_max_f32(lmax);
+        const float nmx = fmaxf(old.x, bmax);
+        float add = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NI; ++i) add += __expf(v[i] - nmx);      // exp(-inf) = 0 for the padding
+        add = warp_sum_f32(add);
+        __syncwarp();
+        if (lane == 0) *ms = make_float2(nmx, old.y * __expf(old.x - nmx) + add);
+    }
+    if (!__any_sync(0xFFFFFFFFu, lmax > tau)) return tau;
+    float bound = -INFINITY;
+    if (k <= 32) {      // 8 groups of 4 lanes, 16 of 2 or 32 of 1: at least k group maxima, all distinct logits
+        float g = lmax;
+        if (k <= 16) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+        if (k <= 8) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, o));
+        bound = g;
+    }
+    int n = 0;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const bool is_cand = v[i] > tau && v[i] >= bound;
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, is_cand);
+        if (is_cand) cbuf[n + __popc(m & ((1u << lane) - 1u))] = make_key(v[i], col0 + lane + 32 * i);
+        n += __popc(m);
+    }
+    for (int j = lane; j < k; j += 32) cbuf[n + j] = list[j];      // empty slots are 0 and rank last
+    __syncwarp();
+    const int total = n + k;
+    for (int e = lane; e < total; e += 32) {
+        const unsigned long long key = cbuf[e];
+        int rank = 0;
+        for (int f = 0; f < total; ++f) rank += cbuf[f] > key ? 1 : 0;
+        if (key != 0ull && rank < k) list[rank] = key;
+    }
+    __syncwarp();
+    const unsigned long long kth = list[k - 1];
+    __syncwarp();
+    return kth != 0ull ? key_logit(kth) : -INFINITY;
+}
+
 // ------------------------------------------------------------------------------------------
 // Merge of P partial results of one draft row by one warp.  Partial p is a record in shared memory
 // at rec[p * stride]: k keys in descending order (0-padded), then (mx_p, s_p) in slot k.
@@ -332,6 +413,21 @@ __device__ __forceinline__ void warp_select_topk(const unsigned long long* rec, 
     __syncwarp();
 }
 
+// Winner j of draft row m: its target id (the d2t gather), log-prob and draft index.
+__device__ __forceinline__ void write_winner(const HeadOut& o, int m, int j, unsigned long long best, float lse) {
+    const size_t out = (size_t)m * o.k + j;
+    if (best != 0ull) {
+        const int idx = key_index(best);
+        o.target_ids[out] = o.d2t ? __ldg(&o.d2t[idx]) : idx;
+        o.logprobs[out] = key_logit(best) - lse;
+        if (o.draft_ids) o.draft_ids[out] = idx;
+    } else {   // fewer than k candidates exist only if a wait ran out upstream
+        o.target_ids[out] = -1;
+        o.logprobs[out] = -INFINITY;
+        if (o.draft_ids) o.draft_ids[out] = -1;
+    }
+}
+
 // Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
 // Winners are written by the lanes that hold them, so the d2t gathers are one round trip, not k.
 __device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride,
@@ -340,20 +436,133 @@ __device__ inline void merge_row_final(const HeadOut& o, int P, int m, const uns
     const int k = o.k;
     const float2 ms = warp_merge_ms(rec, stride, P, k);
     const float lse = ms.x + __logf(ms.y);
-    warp_select_topk(rec, stride, P, k, cbuf, [&](int j, unsigned long long best) {
-        const size_t out = (size_t)m * k + j;
-        if (best != 0ull) {
-            const int idx = key_index(best);
-            o.target_ids[out] = o.d2t ? __ldg(&o.d2t[idx]) : idx;
-            o.logprobs[out] = key_logit(best) - lse;
-            if (o.draft_ids) o.draft_ids[out] = idx;
-        } else {   // fewer than k candidates exist only if a wait ran out upstream
-            o.target_ids[out] = -1;
-            o.logprobs[out] = -INFINITY;
-            if (o.draft_ids) o.draft_ids[out] = -1;
-        }
-    });
+    warp_select_topk(rec, stride, P, k, cbuf, [&](int j, unsigned long long best) { write_winner(o, m, j, best, lse); });
     if (lane == 0 && o.lse) o.lse[m] = lse;
+}
+
+// Row-wise final merge by one warp, straight from the row-major records in global memory (VT_ROW_*), for the
+// warp that published draft row m last.  Three dependent round trips to L2 instead of a staged copy:
+//   1. every CTA's best key and (max, sum-exp): two coalesced reads per lane and 32 CTAs; the log-sum-exp and
+//      the bound of warp_select_topk (smallest of G >= k group maxima) follow from them in registers;
+//   2. only lists whose head reaches the bound can hold a winner (typically one or two dozen of 148): their
+//      deeper keys are fetched in one sweep, the ones at or above the bound join the heads in `cbuf`;
+//   3. rank counting picks the winners; the lanes holding them gather d2t and write the outputs.
+// k > 32, fewer than G lists, or more than `cap` candidates take k rounds of a warp-wide maximum over the list
+// heads instead.  `ql` holds kMaxParts list numbers.  Reads bypass L1: the records were written by other SMs.
+__device__ inline void merge_row_global(const HeadOut& o, int P, int m, unsigned long long* cbuf, int cap,
+                                        unsigned short* ql) {
+    const int lane = threadIdx.x & 31;
+    const int k = o.k, km1 = o.k - 1;
+    const unsigned long long* heads = VT_ROW_HEADS(o, m);
+    const unsigned long long* msr = VT_ROW_MS(o, m);
+    unsigned long long hk[kMergeSlots];
+    float2 ms[kMergeSlots];
+#pragma unroll
+    for (int q = 0; q < kMergeSlots; ++q) {
+        const int p = lane + 32 * q;
+        hk[q] = p < P ? __ldcg(heads + p) : 0ull;
+        ms[q] = p < P ? unpack_ms(__ldcg(msr + p)) : make_float2(-INFINITY, 0.0f);
+    }
+    float mx = -INFINITY;
+    uint32_t lhead = 0u;
+#pragma unroll
+    for (int q = 0; q < kMergeSlots; ++q) {
+        mx = fmaxf(mx, ms[q].x);
+        lhead = max(lhead, (uint32_t)(hk[q] >> 32));
+    }
+    mx = warp_max_f32(mx);
+    float s = 0.0f;
+#pragma unroll
+    for (int q = 0; q < kMergeSlots; ++q)
+        if (ms[q].y > 0.0f) s += ms[q].y * __expf(ms[q].x - mx);
+    s = warp_sum_f32(s);
+    const float lse = mx + __logf(s);
+    if (lane == 0 && o.lse) o.lse[m] = lse;
+
+    bool fast = k <= 32;
+    int n = 0;
+    if (fast) {
+        const int G = k <= 8 ? 8 : k <= 16 ? 16 : 32;
+        const unsigned int have = __ballot_sync(0xFFFFFFFFu, lhead != 0u);
+        const int nvalid = __popc(have);
+        const unsigned int src = __fns(have, 0, lane + 1);
+        uint32_t v = __shfl_sync(0xFFFFFFFFu, lhead, src & 31);
+        if (lane >= nvalid) v = 0u;
+        fast = nvalid >= G;
+        if (G <= 16) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 16));
+        if (G <= 8) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 8));
+        const uint32_t bound = __reduce_min_sync(0xFFFFFFFFu, lane < G ? v : 0xFFFFFFFFu);
+        if (fast) {
+            int nl = 0;                                          // lists whose head reaches the bound
+#pragma unroll
+            for (int q = 0; q < kMergeSlots; ++q) {
+                const bool is_cand = hk[q] != 0ull && (uint32_t)(hk[q] >> 32) >= bound;
+                const unsigned int bm = __ballot_sync(0xFFFFFFFFu, is_cand);
+                if (is_cand) {
+                    const int pos = nl + __popc(bm & ((1u << lane) - 1u));
+                    ql[pos] = (unsigned short)(lane + 32 * q);
+                    if (pos < cap) cbuf[pos] = hk[q];
+                }
+                nl += __popc(bm);
+            }
+            n = nl;
+            fast = nl <= cap;
+            __syncwarp();
+            const int items = nl * km1;
+            for (int base = 0; base < items && fast; base += 128) {
+                unsigned long long key[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e = base + 32 * u + lane;
+                    key[u] = e < items ? __ldcg(VT_ROW_REST(o, m, ql[e / km1]) + e % km1) : 0ull;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool is_cand = key[u] != 0ull && (uint32_t)(key[u] >> 32) >= bound;
+                    const unsigned int bm = __ballot_sync(0xFFFFFFFFu, is_cand);
+                    if (n + __popc(bm) > cap) fast = false;
+                    if (is_cand && fast) cbuf[n + __popc(bm & ((1u << lane) - 1u))] = key[u];
+                    n += __popc(bm);
+                }
+            }
+            __syncwarp();
+        }
+    }
+    if (fast) {
+        for (int e = lane; e < n; e += 32) {
+            const unsigned long long key = cbuf[e];
+            int rank = 0;
+#pragma unroll 4
+            for (int f = 0; f < n; ++f) rank += cbuf[f] > key ? 1 : 0;
+            if (rank < k) write_winner(o, m, rank, key, lse);
+        }
+        for (int j = n + lane; j < k; j += 32) write_winner(o, m, j, 0ull, lse);   // fewer than k keys exist at all
+    } else {
+        // every list descends, so its best remaining key is its head: k rounds of a warp-wide maximum
+        int head[kMergeSlots];
+        unsigned long long local = 0ull;
+#pragma unroll
+        for (int q = 0; q < kMergeSlots; ++q) {
+            head[q] = 0;
+            local = hk[q] > local ? hk[q] : local;
+        }
+        for (int j = 0; j < k; ++j) {
+            const unsigned long long best = warp_max_key(local);
+            if (best != 0ull && local == best) {          // the one lane whose head won advances that list
+                local = 0ull;
+#pragma unroll
+                for (int q = 0; q < kMergeSlots; ++q) {
+                    if (hk[q] == best) {
+                        ++head[q];
+                        hk[q] = head[q] < k ? __ldcg(VT_ROW_REST(o, m, lane + 32 * q) + head[q] - 1) : 0ull;
+                    }
+                    local = hk[q] > local ? hk[q] : local;
+                }
+            }
+            if (lane == (j & 31)) write_winner(o, m, j, best, lse);
+        }
+    }
+    __syncwarp();
 }
 
 // Publishes this CTA's records (already written to global memory by the calling threads) and

@@ -18,11 +18,11 @@
 
 #include "vt_common.cuh"
 #include "vt_launch.h"
+#include "vt_tc.cuh"
 
 namespace vt {
 
 constexpr int kMmaThreads = 384;               // warps 0-3 epilogue, 4 TMA, 5 MMA; the rest only join the final merge
-constexpr int kBoxK = 64;                    // bf16 elements per k-step = one 128-byte swizzle row
 constexpr int kMaxStages = 32;
 constexpr size_t kResidentHMax = 96 * 1024;   // h stays in shared memory when its A blocks fit in this
 constexpr int kAccStride = 256;              // TMEM columns between the two accumulator buffers
@@ -47,120 +47,8 @@ struct MmaParams {
     uint32_t list_off, bar_off, total_smem;   // offsets from the 1024-aligned base
 };
 
-// ------------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128-byte swizzled
-// (the layout a TMA box of 64 bf16 columns writes): 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t desc = 0;
-    desc |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-    desc |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle): 1
-    desc |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
-    desc |= (uint64_t)1 << 46;                           // descriptor version of sm_100
-    desc |= (uint64_t)2 << 61;                           // 128-byte swizzle
-    return desc;
-}
-
 // ------------------------------------------------------------------------------------------ kernel
 constexpr int kMaxBatchCols = 256;            // vocabulary columns the top-k selection takes at a time
-
-// Top-k update of one draft row by a whole warp.  `vals` is the row's logits for `ncols` consecutive
-// vocabulary columns (first column = vocabulary row `col0`), in shared memory; `list` is the row's k best
-// so far (descending keys, 0 = empty) and `tau` the logit of its k-th best (-inf while the list is not
-// full).  Lane L looks at columns L, L+32, ...
-//   1. bound: the 32 lanes form 8, 16 or 32 groups (whichever is >= k; k <= 32); the smallest group maximum
-//      has at least k logits at or above it, so nothing below it can be among the k best of these columns;
-//   2. the logits above tau (strictly: a later row loses a tie) and not below the bound are the candidates;
-//      a ballot per column group gives each its slot in `cbuf`, and the current list follows them;
-//   3. every entry of cbuf counts the entries larger than itself - its rank - and the entries of rank < k
-//      form the new list.  Keys are distinct, so ranks are too.  No step depends on the previous candidate,
-//      unlike an insertion loop.
-// The same pass folds the columns into the row's running (max, sum-exp) in *ms.
-// Returns the new tau.  All lanes must call it; `cbuf` holds kMaxBatchCols + k keys.
-__device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, int col0, unsigned long long* list,
-                                                  int k, float tau, unsigned long long* cbuf, float2* ms, int lane) {
-    constexpr int NI = kMaxBatchCols / 32;
-    float v[NI];
-    float lmax = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const int c = lane + 32 * i;
-        v[i] = c < ncols ? vals[c] : -INFINITY;
-        lmax = fmaxf(lmax, v[i]);
-    }
-    {   // running log-sum-exp of the row: (max, sum of exp(x - max)), folded over these columns by the warp
-        const float2 old = *ms;
-        const float bmax = warp_max_f32(lmax);
-        const float nmx = fmaxf(old.x, bmax);
-        float add = 0.0f;
-#pragma unroll
-        for (int i = 0; i < NI; ++i) add += __expf(v[i] - nmx);      // exp(-inf) = 0 for the padding
-        add = warp_sum_f32(add);
-        __syncwarp();
-        if (lane == 0) *ms = make_float2(nmx, old.y * __expf(old.x - nmx) + add);
-    }
-    if (!__any_sync(0xFFFFFFFFu, lmax > tau)) return tau;
-    float bound = -INFINITY;
-    if (k <= 32) {      // 8 groups of 4 lanes, 16 of 2 or 32 of 1: at least k group maxima, all distinct logits
-        float g = lmax;
-        if (k <= 16) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
-        if (k <= 8) g = fmaxf(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) g = fminf(g, __shfl_xor_sync(0xFFFFFFFFu, g, o));
-        bound = g;
-    }
-    int n = 0;
-#pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const bool is_cand = v[i] > tau && v[i] >= bound;
-        const unsigned int m = __ballot_sync(0xFFFFFFFFu, is_cand);
-        if (is_cand) cbuf[n + __popc(m & ((1u << lane) - 1u))] = make_key(v[i], col0 + lane + 32 * i);
-        n += __popc(m);
-    }
-    for (int j = lane; j < k; j += 32) cbuf[n + j] = list[j];      // empty slots are 0 and rank last
-    __syncwarp();
-    const int total = n + k;
-    for (int e = lane; e < total; e += 32) {
-        const unsigned long long key = cbuf[e];
-        int rank = 0;
-        for (int f = 0; f < total; ++f) rank += cbuf[f] > key ? 1 : 0;
-        if (key != 0ull && rank < k) list[rank] = key;
-    }
-    __syncwarp();
-    const unsigned long long kth = list[k - 1];
-    __syncwarp();
-    return kth != 0ull ? key_logit(kth) : -INFINITY;
-}
 
 // Epilogue in two layouts.  tcgen05.ld gives lane = draft row, registers = 32 consecutive vocabulary
 // logits: the running (max, sum-exp) is kept there, thread-private.  For the top-k the logits are turned
@@ -399,7 +287,7 @@ head_mma_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__
                 const int bcol0 = row0 + c0 - cb;                              // vocabulary row of its first column
                 for (int m = member; m < p.m_count; m += team) {
                     const float* vals = tiles + (size_t)(m >> 5) * p.tile_floats + (size_t)(m & 31) * EBP;
-                    const float t2 = warp_topk_update(vals, bvalid, bcol0, epi + (size_t)m * k, k, thr_s[m], cbuf,
+                    const float t2 = warp_topk_update<kMaxBatchCols / 32>(vals, bvalid, bcol0, epi + (size_t)m * k, k, thr_s[m], cbuf,
                                                       ms_s + m, lane);
                     if (lane == 0) thr_s[m] = t2;
                 }
@@ -459,7 +347,7 @@ static vt_status get_encode(EncodeTiledFn* out) {
 }
 
 // bf16 matrix [rows, d] row-major, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
-static vt_status make_map(CUtensorMap* map, const void* ptr, int rows, int d, int box_rows) {
+vt_status make_tensor_map_bf16(CUtensorMap* map, const void* ptr, int rows, int d, int box_rows) {
     EncodeTiledFn enc;
     vt_status r = get_encode(&enc);
     if (r != VT_OK) return r;
@@ -511,13 +399,13 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
     }
 
     CUtensorMap tmW;
-    r = make_map(&tmW, c.W, c.Vt, c.d, NT);
+    r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, NT);
     if (r != VT_OK) return r;
 
     for (int m0 = 0; m0 < c.M; m0 += 128) {
         const int mc = std::min(128, c.M - m0);
         CUtensorMap tmH;
-        r = make_map(&tmH, c.h, c.M, c.d, mc);
+        r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, mc);
         if (r != VT_OK) return r;
 
         MmaParams p{};

@@ -1,0 +1,371 @@
+// Draft head, tensor-core path for few draft rows (M <= 16): vocabulary rows on the TMEM lanes.
+//
+//   D[i, m] = sum_j W_trim[row0 + i, j] * h[m, j]       (the d -> k linear head, 2*d*k FLOPs per draft row)
+//
+// Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (16 rows: the
+// draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes x 16 columns in tensor
+// memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
+// row, so reading a tile out costs one instruction per thread whatever M is, and a weight tile needs no
+// padding rows: the tile height is the CTA's row count split evenly (<= 128), rows of the MMA past it compute
+// on stale shared memory and land in lanes nobody reads.  h stays in shared memory for the whole kernel.
+//   warp 8     TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
+//   warp 9     MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
+//              ring stage; two accumulator buffers in TMEM
+//   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory
+//   warps 0-7  warp w owns draft rows w and w+8: running (max, sum-exp) and top-k of the row over the tile
+//              (warp_topk_update), and at the end the row's record, its arrival ticket and, for the warp that
+//              arrives last of all CTAs, the row's final merge (merge_row_global).  No CTA-wide barrier and no
+//              CTA ever waits for another.
+// The weight stream is the bound (arithmetic intensity = M FLOP/B).
+#include <cuda.h>
+
+#include "vt_common.cuh"
+#include "vt_launch.h"
+#include "vt_tc.cuh"
+
+namespace vt {
+
+constexpr int kSmThreads = 320;
+constexpr int kSmEpiWarps = 8;                // warps 0-7; warps 0-3 also read TMEM
+constexpr int kSmProducerWarp = 8, kSmMmaWarp = 9;
+constexpr int kSmMaxM = 16;                   // draft rows = MMA N
+constexpr int kSmMaxStages = 32;
+constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
+constexpr int kHParts = 4;                    // h arrives in this many parts so the first MMAs need not wait for all of it
+constexpr int kSmCand = 128 + VT_MAX_K;       // candidate keys per epilogue warp (one tile's columns + the list)
+constexpr uint32_t kSmScratch = kSmCand * 8 + kMaxParts * 2;   // per warp: candidates, then list numbers for the merge
+
+struct SmallParams {
+    HeadOut out;
+    int M;                    // draft rows, <= kSmMaxM
+    int d, nk;                // nk = 64-column k-blocks
+    int TH;                   // vocabulary rows per tile (<= 128)
+    int kb_per_stage;         // k-blocks one ring stage holds
+    int n_stages;
+    uint32_t slot_bytes;      // one k-block of a tile in the ring: TH rounded up to whole 8-row groups x 128 B
+    uint32_t stage_bytes;
+    uint32_t w_tx;            // bytes one W box delivers (TH * 128)
+    uint32_t h_blk;           // bytes of one k-block of h: 8 or 16 rows x 128 B
+    uint32_t h_off, lg_off, list_off, scratch_off, bar_off, total_smem;   // from the 1024-aligned base
+    uint32_t idesc;
+};
+
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+// Barrier among the epilogue warps only (the producer and the MMA issuer never join it).
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kSmEpiWarps * 32) : "memory"); }
+
+__global__ void __launch_bounds__(kSmThreads, 1)
+head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
+                      const SmallParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (base - raw);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int Vt = p.out.Vt, k = p.out.k, M = p.M, TH = p.TH, S = p.n_stages, nk = p.nk;
+    const int row_begin = (int)((long long)cta * Vt / G);
+    const int row_end = (int)((long long)(cta + 1) * Vt / G);
+    const int nrows = row_end - row_begin;
+    const int ntiles = (nrows + TH - 1) / TH;
+    const int h_part = (nk + kHParts - 1) / kHParts;          // k-blocks per part of h
+
+    float* lg = reinterpret_cast<float*>(smem + p.lg_off);                                  // [M][kLgPitch]
+    unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [M][k]
+    float2* ms_s = reinterpret_cast<float2*>(lists + (size_t)M * k);                         // [kSmMaxM]
+    unsigned char* scratch = smem + p.scratch_off + (uint32_t)(warp & 7) * kSmScratch;
+    const uint32_t bar_full = base + p.bar_off, bar_empty = bar_full + 8u * S;
+    const uint32_t bar_accf = bar_empty + 8u * S, bar_acce = bar_accf + 16u;
+    const uint32_t bar_h = bar_acce + 16u, bar_drain = bar_h + 8u * kHParts;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + p.bar_off + 8u * (2 * S + 4 + kHParts + 1));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    if (warp == kSmProducerWarp && lane == 0) {      // descriptor fetches overlap the barrier set-up below
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
+    }
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_accf + 8u * b, 1);
+            mbar_init(bar_acce + 8u * b, 4);
+        }
+        for (int j = 0; j < kHParts; ++j) mbar_init(bar_h + 8u * j, 1);
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    for (int i = tid; i < M * k; i += blockDim.x) lists[i] = 0ull;
+    if (tid < kSmMaxM) ms_s[tid] = make_float2(-INFINITY, 0.0f);
+    // With 8 rows of h per k-block the MMA's rows 8-15 alias the next k-block; the last one reads this pad.
+    for (int i = tid; i < 256; i += blockDim.x)
+        reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
+    if (warp == kSmMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(32u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // everything above touched only shared memory, tensor memory and kernel parameters
+    grid_dependency_wait();
+    if (tid == 0) grid_launch_dependents();
+    fence_proxy_async();          // the zeroed pad is read by the tensor core (async proxy)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto fail = [&]() {
+        *abort_flag = 1;
+        atomicOr(&p.out.hdr->status, kStatusTimeout);
+    };
+
+    if (warp == kSmProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer: the weight stream
+        if (lane == 0) {
+            int s = 0, issued = 0;
+            uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
+            bool ok = true;
+            const int kbs = p.kb_per_stage;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int row0 = row_begin + t * TH;
+                for (int ks = 0; ks < nk; ks += kbs) {
+                    if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
+                    if (*abort_flag) { ok = false; break; }
+                    const int nb = min(kbs, nk - ks);
+                    const uint32_t bar = bar_full + 8u * s;
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * p.w_tx);
+                    for (int kb = 0; kb < nb; ++kb)
+                        tma_load_2d(base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.slot_bytes, &tmW,
+                                    (ks + kb) * kBoxK, row0, bar);
+                    ++issued;
+                    if (++s == S) { s = 0; ++wrap; }
+                }
+            }
+            if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
+                for (int i = max(0, issued - S); i < issued; ++i)
+                    (void)mbar_wait(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u);
+            }
+        }
+    } else if (warp == kSmMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            const uint64_t desc0 = smem_desc_sw128(base);                      // descriptor of the ring's first byte
+            const uint64_t h_desc0 = smem_desc_sw128(base + p.h_off);
+            const uint32_t stage_units = p.stage_bytes >> 4, slot_units = p.slot_bytes >> 4, h_units = p.h_blk >> 4;
+            const int kbs = p.kb_per_stage;
+            int h_ready = 0;                                                   // k-blocks of h known to have landed
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int buf = t & 1;
+                if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 16);
+                for (int ks = 0; ks < nk && ok; ks += kbs) {
+                    const int nb = min(kbs, nk - ks);
+                    while (h_ready < ks + nb) {
+                        if (!mbar_wait(bar_h + 8u * (uint32_t)(h_ready / h_part), 0u)) { fail(); ok = false; break; }
+                        h_ready += h_part;
+                    }
+                    if (!ok) break;
+                    if (!mbar_wait(bar_full + 8u * s, phase)) { fail(); ok = false; break; }
+                    if (*abort_flag) { ok = false; break; }
+                    tc_fence_after();
+                    for (int kb = 0; kb < nb; ++kb) {
+                        const uint64_t a_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * slot_units);
+                        const uint64_t b_desc = h_desc0 + (uint64_t)((uint32_t)(ks + kb) * h_units);
+                        // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
+                        tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                    }
+                    tc_commit(bar_empty + 8u * s);
+                    if (++s == S) { s = 0; phase ^= 1u; }
+                }
+                if (ok) tc_commit(bar_accf + 8u * buf);
+            }
+            if (*abort_flag) {   // every MMA issued so far must retire before TMEM is freed
+                tc_commit(bar_drain);
+                (void)mbar_wait(bar_drain, 0u);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps 0-7
+        if (warp == kSmEpiWarps - 1 && lane == 0 && ntiles > 0) {
+            // h, fetched once: every CTA needs all of it, one box per k-block, in kHParts parts
+            for (int j = 0; j < kHParts; ++j) {
+                const int k0 = j * h_part, k1 = min(nk, k0 + h_part);
+                if (k0 >= k1) break;
+                mbar_arrive_expect_tx(bar_h + 8u * j, (uint32_t)(k1 - k0) * p.h_blk);
+                for (int kb = k0; kb < k1; ++kb)
+                    tma_load_2d(base + p.h_off + (uint32_t)kb * p.h_blk, &tmH, kb * kBoxK, 0, bar_h + 8u * j);
+            }
+        }
+        __syncwarp();
+        unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(scratch);
+        float tau[2] = {-INFINITY, -INFINITY};
+        // Every epilogue warp passes the same two barriers per tile whatever happens, so none can be left
+        // waiting at one: after a wait has run out the remaining tiles only skip their work.
+        for (int t = 0; t < ntiles; ++t) {
+            const int buf = t & 1;
+            const int row0 = row_begin + t * TH;
+            const int nv = min(TH, row_end - row0);
+            if (warp < 4) {
+                // warp-uniform decisions: tcgen05.ld needs the whole warp
+                bool got = false;
+                if (!__any_sync(0xFFFFFFFFu, *abort_flag != 0)) {
+                    got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u));
+                    if (!got) fail();
+                }
+                if (got) {
+                    tc_fence_after();
+                    uint32_t r[16];
+                    tc_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 16), r);
+                    tc_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                    const int i = warp * 32 + lane;                    // TMEM lane = vocabulary row of the tile
+                    if (i < nv) {
+#pragma unroll
+                        for (int m = 0; m < kSmMaxM; ++m)
+                            if (m < M) lg[m * kLgPitch + i] = __uint_as_float(r[m]);
+                        if (p.out.logits) {
+#pragma unroll
+                            for (int m = 0; m < kSmMaxM; ++m)
+                                if (m < M) p.out.logits[(size_t)m * Vt + row0 + i] = __uint_as_float(r[m]);
+                        }
+                    }
+                }
+            }
+            epi_barrier();                                             // the tile's logits are in shared memory
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int m = warp + kSmEpiWarps * q;
+                if (m < M)
+                    tau[q] = warp_topk_update<4>(lg + m * kLgPitch, nv, row0, lists + (size_t)m * k, k, tau[q], cbuf,
+                                                 ms_s + m, lane);
+            }
+            epi_barrier();                                             // ... and may be overwritten
+        }
+        // ------------------------------------------------------------------ publish, and merge if last
+        // The warp owns its rows from the first tile to the outputs: record -> fence -> ticket; the warp that
+        // draws the last ticket of a row (over all CTAs) merges that row.  No CTA-wide step in between.
+        for (int m = warp; m < M; m += kSmEpiWarps) {
+            const unsigned long long* list = lists + (size_t)m * k;
+            for (int j = lane; j < k; j += 32) {
+                if (j == 0) VT_ROW_HEADS(p.out, m)[cta] = list[0];
+                else VT_ROW_REST(p.out, m, cta)[j - 1] = list[j];
+            }
+            if (lane == 0) {
+                const float2 ms = ms_s[m];
+                VT_ROW_MS(p.out, m)[cta] = pack_ms(ms.x, ms.y);
+            }
+            __threadfence();
+            __syncwarp();
+            unsigned int ticket = 0;
+            if (lane == 0) ticket = atomicAdd(&p.out.hdr->row_ticket[m], 1u);
+            ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+            if (ticket == (unsigned int)G - 1u) {
+                __threadfence();
+                merge_row_global(p.out, G, m, cbuf, kSmCand, reinterpret_cast<unsigned short*>(scratch + kSmCand * 8));
+                if (lane == 0) p.out.hdr->row_ticket[m] = 0u;          // ready for the next call
+            }
+        }
+        if (warp == kSmEpiWarps - 1 && lane == 0 && ntiles > 0 && *abort_flag) {
+            // let the copies of h land before the CTA gives its shared memory back
+            for (int j = 0; j < kHParts && j * h_part < nk; ++j) (void)mbar_wait(bar_h + 8u * j, 0u);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kSmMmaWarp)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32u) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------ host
+// Shared memory the kernel needs beside the ring, and the tile geometry, for a shape; false if h does not fit.
+static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
+    if (M < 1 || M > kSmMaxM) return false;
+    const int R = (Vt + grid - 1) / grid;                    // most rows a CTA owns
+    const int nt = (R + 127) / 128;
+    p->M = M;
+    p->d = d;
+    p->nk = (d + kBoxK - 1) / kBoxK;
+    p->TH = (R + nt - 1) / nt;
+    p->w_tx = (uint32_t)p->TH * 128u;
+    p->slot_bytes = (uint32_t)((p->TH + 7) / 8) * 1024u;
+    p->h_blk = M <= 8 ? 1024u : 2048u;
+    // a stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height
+    p->kb_per_stage = std::max(1, std::min(std::min(4, p->nk), (int)((28 * 1024 + p->slot_bytes / 2) / p->slot_bytes)));
+    p->stage_bytes = p->slot_bytes * (uint32_t)p->kb_per_stage;
+    // instruction descriptor: D fp32, A and B bf16, both K-major, N = 16, M = 128
+    p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const size_t h_bytes = (size_t)p->nk * p->h_blk + 1024;               // + the pad the last k-block's rows 8-15 read
+    const size_t lg_bytes = (size_t)M * kLgPitch * 4;
+    const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 8) + 127) & ~(size_t)127;
+    const size_t scratch_bytes = ((size_t)kSmEpiWarps * kSmScratch + 127) & ~(size_t)127;
+    const size_t bar_bytes = (size_t)(2 * kSmMaxStages + 4 + kHParts + 1) * 8 + 16;
+    const size_t fixed = 1024 + h_bytes + ((lg_bytes + 127) & ~(size_t)127) + list_bytes + scratch_bytes + bar_bytes + 128;
+    if (fixed + 2 * (size_t)p->stage_bytes > (size_t)kMaxDynSmem) return false;
+    const int S = (int)std::min<size_t>(kSmMaxStages, ((size_t)kMaxDynSmem - fixed) / p->stage_bytes);
+    const size_t ring = (size_t)S * p->stage_bytes;
+    if (S < 3) return false;                                              // too few bytes in flight to be worth it
+    p->n_stages = S;
+    p->h_off = (uint32_t)ring;                                            // stages are multiples of 1024 bytes
+    p->lg_off = (uint32_t)(ring + h_bytes);
+    p->list_off = (uint32_t)(p->lg_off + ((lg_bytes + 127) & ~(size_t)127));
+    p->scratch_off = (uint32_t)(p->list_off + list_bytes);
+    p->bar_off = (uint32_t)(p->scratch_off + scratch_bytes);
+    // An MMA always reads 128 A rows = 16 KB from its slot's first byte: past a short tile that is whatever
+    // follows in shared memory, which must still be inside the allocation.
+    const size_t need = std::max((size_t)p->bar_off + bar_bytes, ring - p->slot_bytes + 16384);
+    p->total_smem = (uint32_t)(need + 1024);
+    return p->total_smem <= (uint32_t)kMaxDynSmem;
+}
+
+vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_out) {
+    int sms = 0;
+    vt_status r = device_sm_count(&sms);
+    if (r != VT_OK) return r;
+    const int grid = head_grid(sms, c.Vt, 16);
+    *grid_out = grid;
+    SmallParams p{};
+    if (!c.out.fused_merge || !small_plan(c.M, c.d, c.Vt, c.out.k, grid, &p)) return VT_ERR_UNSUPPORTED;
+    p.out = c.out;
+
+    static int configured_device = -1;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    if (configured_device != dev) {
+        cudaError_t e = cudaFuncSetAttribute(head_mma_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+        if (e != cudaSuccess) return cuda_fail(e);
+        configured_device = dev;
+    }
+    CUtensorMap tmW, tmH;
+    r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, p.TH);
+    if (r != VT_OK) return r;
+    r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
+    if (r != VT_OK) return r;
+    cudaError_t e = launch_pdl(head_mma_small_kernel, grid, kSmThreads, p.total_smem, st, tmW, tmH, p);
+    count_launch();
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+}  // namespace vt

@@ -1,4 +1,4 @@
-"""Seeded random shapes through both head paths against the oracle: draft-row counts across every per-pass
+"""Seeded random shapes through every head path against the oracle: draft-row counts across every per-pass
 limit (2, 4, 8, 16, 32, 128), vocabulary sizes below and above the CTA count and off every tile size,
 k from 1 to VT_MAX_K, hidden sizes that are not multiples of the 64-column k-block."""
 import numpy as np
@@ -41,6 +41,7 @@ def test_random_shape_both_paths(vt, oracle, M, d, Vt, k):
     h, W, d2t = rand_case(M, d, Vt, seed=M * 31 + d * 7 + Vt + k)
     ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
     Wd = dev_bf16(W)
-    for path in (vt.VT_PATH_AUTO, vt.VT_PATH_GEMV, vt.VT_PATH_MMA):
+    paths = (vt.VT_PATH_AUTO, vt.VT_PATH_GEMV, vt.VT_PATH_MMA) + ((vt.VT_PATH_MMA_SMALL,) if M <= 16 else ())
+    for path in paths:
         got = run_head(vt, h, Wd, d2t, k, path)
         parity.check_head(got, ora, d2t, k)

@@ -31,7 +31,14 @@ def rand_case(M, d, Vt, seed, w_std=0.02, h_std=1.0):
     return h, W, d2t
 
 
-PATHS = [pytest.param(1, id="gemv"), pytest.param(2, id="mma")]
+PATHS = [pytest.param(1, id="gemv"), pytest.param(2, id="mma"), pytest.param(3, id="mma_small")]
+SMALL_MAX_M = 16          # VT_PATH_MMA_SMALL takes at most this many draft rows
+
+
+def skip_unless_path_takes(path, M):
+    if path == 3 and M > SMALL_MAX_M:
+        pytest.skip("the few-draft-rows tensor-core path takes M <= 16")
+
 
 
 # ------------------------------------------------------------------------------ compaction
@@ -112,6 +119,7 @@ LOGIT_SHAPES = [(1, 8, 1), (1, 64, 7), (3, 64, 127), (8, 2048, 129), (2, 3072, 1
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("M,d,Vt", LOGIT_SHAPES)
 def test_logits_vs_oracle(vt, oracle, path, M, d, Vt):
+    skip_unless_path_takes(path, M)
     h, W, _ = rand_case(M, d, Vt, seed=M * 1000 + Vt)
     got = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=path).cpu().numpy()
     parity.check_logits(got, oracle.logits(h, W))
@@ -120,12 +128,14 @@ def test_logits_vs_oracle(vt, oracle, path, M, d, Vt):
 # ------------------------------------------------------------------------------ full head
 HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8), (8, 2048, 129, 10),
                (8, 4096, 6521, 8), (2, 3072, 1000, 64), (9, 2048, 300, 10), (17, 128, 1025, 3),
-               (4, 5120, 700, 8), (64, 512, 333, 10), (5, 200, 2000, 33), (1, 4096, 13264, 1)]
+               (4, 5120, 700, 8), (64, 512, 333, 10), (5, 200, 2000, 33), (1, 4096, 13264, 1),
+               (16, 256, 40000, 10), (7, 64, 60001, 64), (12, 4096, 3000, 8), (2, 8192, 600, 5)]
 
 
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("M,d,Vt,k", HEAD_SHAPES)
 def test_draft_head_vs_oracle(vt, oracle, path, M, d, Vt, k):
+    skip_unless_path_takes(path, M)
     h, W, d2t = rand_case(M, d, Vt, seed=M * 77 + Vt + k)
     ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
     got = run_head(vt, h, dev_bf16(W), d2t, k, path)
@@ -184,11 +194,19 @@ def test_same_input_twice_is_bit_identical_and_workspace_is_reusable(vt, oracle,
     parity.check_head(got, oracle.draft_head(h2, W2, d2t2, 3, want_logits=True), d2t2, 3)
 
 
-def test_both_paths_agree_on_logits(vt):
+def test_all_paths_agree_on_logits(vt):
     h, W, _ = rand_case(8, 4096, 2000, seed=11)
     a = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=1).cpu().numpy()
     b = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=2).cpu().numpy()
-    assert np.max(np.abs(a - b)) <= 2e-3
+    c = vt.vt_debug_logits(dev_bf16(h), dev_bf16(W), path=3).cpu().numpy()
+    assert np.max(np.abs(a - b)) <= 2e-3 and np.max(np.abs(a - c)) <= 2e-3
+
+
+def test_forced_small_path_refuses_many_draft_rows(vt):
+    h, W, d2t = rand_case(17, 64, 100, seed=12)
+    with pytest.raises(vt.VtError) as e:
+        run_head(vt, h, dev_bf16(W), d2t, 4, 3)
+    assert e.value.status == vt.VT_ERR_UNSUPPORTED
 
 
 def test_trimmed_head_equals_full_head_restricted(vt, oracle):
