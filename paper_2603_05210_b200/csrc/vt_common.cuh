@@ -51,13 +51,11 @@ __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
 
 // Row-major records (the row-wise merge of the few-draft-rows kernel): draft row m owns kMaxParts * (k + 1)
 // consecutive u64 of the same record area,
-//   heads [kMaxParts]          every CTA's best key        (one coalesced read finds the lists that matter)
-//   ms    [kMaxParts]          every CTA's (max, sum-exp)
-//   rest  [kMaxParts][k - 1]   every CTA's 2nd .. k-th key
+//   ms   [kMaxParts]        every CTA's (max, sum-exp)
+//   keys [k][kMaxParts]     keys[j][p] = CTA p's j-th best key: one coalesced read per depth
 // M * kMaxParts * (k + 1) <= kMaxParts * ws_pitch(M, k), so the area vt_workspace_bytes sizes holds either layout.
-#define VT_ROW_HEADS(o, m) ((o).recs + (size_t)(m) * kMaxParts * ((o).k + 1))
-#define VT_ROW_MS(o, m) (VT_ROW_HEADS(o, m) + kMaxParts)
-#define VT_ROW_REST(o, m, p) (VT_ROW_HEADS(o, m) + 2 * kMaxParts + (size_t)(p) * ((o).k - 1))
+#define VT_ROW_MS(o, m) ((o).recs + (size_t)(m) * kMaxParts * ((o).k + 1))
+#define VT_ROW_KEYS(o, m, j) (VT_ROW_MS(o, m) + (size_t)((j) + 1) * kMaxParts)
 
 struct HeadOut {
     const int32_t* d2t;   // null: report draft indices as target ids
@@ -441,128 +439,73 @@ __device__ inline void merge_row_final(const HeadOut& o, int P, int m, const uns
 }
 
 // Row-wise final merge by one warp, straight from the row-major records in global memory (VT_ROW_*), for the
-// warp that published draft row m last.  Three dependent round trips to L2 instead of a staged copy:
-//   1. every CTA's best key and (max, sum-exp): two coalesced reads per lane and 32 CTAs; the log-sum-exp and
-//      the bound of warp_select_topk (smallest of G >= k group maxima) follow from them in registers;
-//   2. only lists whose head reaches the bound can hold a winner (typically one or two dozen of 148): their
-//      deeper keys are fetched in one sweep, the ones at or above the bound join the heads in `cbuf`;
-//   3. rank counting picks the winners; the lanes holding them gather d2t and write the outputs.
-// k > 32, fewer than G lists, or more than `cap` candidates take k rounds of a warp-wide maximum over the list
-// heads instead.  `ql` holds kMaxParts list numbers.  Reads bypass L1: the records were written by other SMs.
-__device__ inline void merge_row_global(const HeadOut& o, int P, int m, unsigned long long* cbuf, int cap,
-                                        unsigned short* ql) {
+// warp that published draft row m last.  One round trip to L2 brings every CTA's (max, sum-exp) and its three
+// best keys into registers (lane L owns CTAs L, L+32, ...); the log-sum-exp follows from the former.  Every list
+// descends, so its best remaining key is its head: k rounds of a warp-wide maximum over the heads pick the
+// winners in order, and the lane whose head won moves on to that list's next key - from its registers, or,
+// for the rare list that places more than three winners, with one more load.  The lanes holding the winners
+// gather d2t and write the outputs together.  Reads bypass L1: the records were written by other SMs.
+template <int SLOTS>
+__device__ __forceinline__ void merge_row_global_n(const HeadOut& o, int P, int m) {
+    constexpr int kPre = 3;
     const int lane = threadIdx.x & 31;
-    const int k = o.k, km1 = o.k - 1;
-    const unsigned long long* heads = VT_ROW_HEADS(o, m);
+    const int k = o.k;
     const unsigned long long* msr = VT_ROW_MS(o, m);
-    unsigned long long hk[kMergeSlots];
-    float2 ms[kMergeSlots];
+    unsigned long long pre[kPre][SLOTS];
+    float2 ms[SLOTS];
 #pragma unroll
-    for (int q = 0; q < kMergeSlots; ++q) {
+    for (int q = 0; q < SLOTS; ++q) {
         const int p = lane + 32 * q;
-        hk[q] = p < P ? __ldcg(heads + p) : 0ull;
         ms[q] = p < P ? unpack_ms(__ldcg(msr + p)) : make_float2(-INFINITY, 0.0f);
+#pragma unroll
+        for (int j = 0; j < kPre; ++j) pre[j][q] = (p < P && j < k) ? __ldcg(VT_ROW_KEYS(o, m, j) + p) : 0ull;
     }
     float mx = -INFINITY;
-    uint32_t lhead = 0u;
 #pragma unroll
-    for (int q = 0; q < kMergeSlots; ++q) {
-        mx = fmaxf(mx, ms[q].x);
-        lhead = max(lhead, (uint32_t)(hk[q] >> 32));
-    }
+    for (int q = 0; q < SLOTS; ++q) mx = fmaxf(mx, ms[q].x);
     mx = warp_max_f32(mx);
     float s = 0.0f;
 #pragma unroll
-    for (int q = 0; q < kMergeSlots; ++q)
+    for (int q = 0; q < SLOTS; ++q)
         if (ms[q].y > 0.0f) s += ms[q].y * __expf(ms[q].x - mx);
     s = warp_sum_f32(s);
     const float lse = mx + __logf(s);
     if (lane == 0 && o.lse) o.lse[m] = lse;
 
-    bool fast = k <= 32;
-    int n = 0;
-    if (fast) {
-        const int G = k <= 8 ? 8 : k <= 16 ? 16 : 32;
-        const unsigned int have = __ballot_sync(0xFFFFFFFFu, lhead != 0u);
-        const int nvalid = __popc(have);
-        const unsigned int src = __fns(have, 0, lane + 1);
-        uint32_t v = __shfl_sync(0xFFFFFFFFu, lhead, src & 31);
-        if (lane >= nvalid) v = 0u;
-        fast = nvalid >= G;
-        if (G <= 16) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 16));
-        if (G <= 8) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 8));
-        const uint32_t bound = __reduce_min_sync(0xFFFFFFFFu, lane < G ? v : 0xFFFFFFFFu);
-        if (fast) {
-            int nl = 0;                                          // lists whose head reaches the bound
+    int depth[SLOTS];
+    unsigned long long cur[SLOTS];
+    unsigned long long local = 0ull, mine0 = 0ull, mine1 = 0ull;   // winners lane and lane + 32
 #pragma unroll
-            for (int q = 0; q < kMergeSlots; ++q) {
-                const bool is_cand = hk[q] != 0ull && (uint32_t)(hk[q] >> 32) >= bound;
-                const unsigned int bm = __ballot_sync(0xFFFFFFFFu, is_cand);
-                if (is_cand) {
-                    const int pos = nl + __popc(bm & ((1u << lane) - 1u));
-                    ql[pos] = (unsigned short)(lane + 32 * q);
-                    if (pos < cap) cbuf[pos] = hk[q];
-                }
-                nl += __popc(bm);
-            }
-            n = nl;
-            fast = nl <= cap;
-            __syncwarp();
-            const int items = nl * km1;
-            for (int base = 0; base < items && fast; base += 128) {
-                unsigned long long key[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int e = base + 32 * u + lane;
-                    key[u] = e < items ? __ldcg(VT_ROW_REST(o, m, ql[e / km1]) + e % km1) : 0ull;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const bool is_cand = key[u] != 0ull && (uint32_t)(key[u] >> 32) >= bound;
-                    const unsigned int bm = __ballot_sync(0xFFFFFFFFu, is_cand);
-                    if (n + __popc(bm) > cap) fast = false;
-                    if (is_cand && fast) cbuf[n + __popc(bm & ((1u << lane) - 1u))] = key[u];
-                    n += __popc(bm);
-                }
-            }
-            __syncwarp();
-        }
+    for (int q = 0; q < SLOTS; ++q) {
+        depth[q] = 0;
+        cur[q] = pre[0][q];
+        local = cur[q] > local ? cur[q] : local;
     }
-    if (fast) {
-        for (int e = lane; e < n; e += 32) {
-            const unsigned long long key = cbuf[e];
-            int rank = 0;
-#pragma unroll 4
-            for (int f = 0; f < n; ++f) rank += cbuf[f] > key ? 1 : 0;
-            if (rank < k) write_winner(o, m, rank, key, lse);
-        }
-        for (int j = n + lane; j < k; j += 32) write_winner(o, m, j, 0ull, lse);   // fewer than k keys exist at all
-    } else {
-        // every list descends, so its best remaining key is its head: k rounds of a warp-wide maximum
-        int head[kMergeSlots];
-        unsigned long long local = 0ull;
+    for (int j = 0; j < k; ++j) {
+        const unsigned long long best = warp_max_key(local);
+        if (best != 0ull && local == best) {          // keys are unique: exactly one lane, one list
+            local = 0ull;
 #pragma unroll
-        for (int q = 0; q < kMergeSlots; ++q) {
-            head[q] = 0;
-            local = hk[q] > local ? hk[q] : local;
-        }
-        for (int j = 0; j < k; ++j) {
-            const unsigned long long best = warp_max_key(local);
-            if (best != 0ull && local == best) {          // the one lane whose head won advances that list
-                local = 0ull;
-#pragma unroll
-                for (int q = 0; q < kMergeSlots; ++q) {
-                    if (hk[q] == best) {
-                        ++head[q];
-                        hk[q] = head[q] < k ? __ldcg(VT_ROW_REST(o, m, lane + 32 * q) + head[q] - 1) : 0ull;
-                    }
-                    local = hk[q] > local ? hk[q] : local;
+            for (int q = 0; q < SLOTS; ++q) {
+                if (cur[q] == best) {
+                    const int dq = ++depth[q];
+                    cur[q] = dq == 1 ? pre[1][q] : dq == 2 ? pre[2][q]
+                           : dq < k ? __ldcg(VT_ROW_KEYS(o, m, dq) + lane + 32 * q) : 0ull;
                 }
+                local = cur[q] > local ? cur[q] : local;
             }
-            if (lane == (j & 31)) write_winner(o, m, j, best, lse);
         }
+        if (j == lane) mine0 = best;
+        if (j == lane + 32) mine1 = best;
     }
+    if (lane < k) write_winner(o, m, lane, mine0, lse);
+    if (lane + 32 < k) write_winner(o, m, lane + 32, mine1, lse);
     __syncwarp();
+}
+
+__device__ inline void merge_row_global(const HeadOut& o, int P, int m) {
+    if (P <= 160) merge_row_global_n<5>(o, P, m);
+    else merge_row_global_n<kMergeSlots>(o, P, m);
 }
 
 // Publishes this CTA's records (already written to global memory by the calling threads) and

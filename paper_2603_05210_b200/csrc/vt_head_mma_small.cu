@@ -33,7 +33,7 @@ constexpr int kSmMaxStages = 32;
 constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
 constexpr int kHParts = 4;                    // h arrives in this many parts so the first MMAs need not wait for all of it
 constexpr int kSmCand = 128 + VT_MAX_K;       // candidate keys per epilogue warp (one tile's columns + the list)
-constexpr uint32_t kSmScratch = kSmCand * 8 + kMaxParts * 2;   // per warp: candidates, then list numbers for the merge
+constexpr uint32_t kSmScratch = kSmCand * 8;
 
 struct SmallParams {
     HeadOut out;
@@ -116,14 +116,16 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                      ::"r"(smem_u32(tmem_slot)), "r"(32u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // everything above touched only shared memory, tensor memory and kernel parameters
-    grid_dependency_wait();
-    if (tid == 0) grid_launch_dependents();
     fence_proxy_async();          // the zeroed pad is read by the tensor core (async proxy)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above touched only shared memory, tensor memory and kernel parameters, so under programmatic
+    // dependent launch it overlaps the previous kernel's tail.  No thread reads or writes global memory before
+    // this wait (it returns once the previous kernel has completed and its writes are visible).
+    grid_dependency_wait();
+    if (tid == 0) grid_launch_dependents();
 
     auto fail = [&]() {
         *abort_flag = 1;
@@ -137,6 +139,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
             bool ok = true;
             const int kbs = p.kb_per_stage;
+            const uint64_t stream_once = l2_policy_evict_first();
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * TH;
                 for (int ks = 0; ks < nk; ks += kbs) {
@@ -146,8 +149,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     const uint32_t bar = bar_full + 8u * s;
                     mbar_arrive_expect_tx(bar, (uint32_t)nb * p.w_tx);
                     for (int kb = 0; kb < nb; ++kb)
-                        tma_load_2d(base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.slot_bytes, &tmW,
-                                    (ks + kb) * kBoxK, row0, bar);
+                        tma_load_2d_hint(base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.slot_bytes, &tmW,
+                                         (ks + kb) * kBoxK, row0, bar, stream_once);
                     ++issued;
                     if (++s == S) { s = 0; ++wrap; }
                 }
@@ -266,10 +269,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         // draws the last ticket of a row (over all CTAs) merges that row.  No CTA-wide step in between.
         for (int m = warp; m < M; m += kSmEpiWarps) {
             const unsigned long long* list = lists + (size_t)m * k;
-            for (int j = lane; j < k; j += 32) {
-                if (j == 0) VT_ROW_HEADS(p.out, m)[cta] = list[0];
-                else VT_ROW_REST(p.out, m, cta)[j - 1] = list[j];
-            }
+            for (int j = lane; j < k; j += 32) VT_ROW_KEYS(p.out, m, j)[cta] = list[j];
             if (lane == 0) {
                 const float2 ms = ms_s[m];
                 VT_ROW_MS(p.out, m)[cta] = pack_ms(ms.x, ms.y);
@@ -281,7 +281,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
             if (ticket == (unsigned int)G - 1u) {
                 __threadfence();
-                merge_row_global(p.out, G, m, cbuf, kSmCand, reinterpret_cast<unsigned short*>(scratch + kSmCand * 8));
+                merge_row_global(p.out, G, m);
                 if (lane == 0) p.out.hdr->row_ticket[m] = 0u;          // ready for the next call
             }
         }
