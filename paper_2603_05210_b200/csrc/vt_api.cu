@@ -70,10 +70,17 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
     return o;
 }
 
-// M at or below which the vocabulary-rows-on-lanes tensor-core kernel is tried first (it needs h to fit in
-// shared memory), and M at or below which the CUDA-core GEMV comes next.
+// Automatic path choice, from measurements at d = 4096 over V_trim = 4096 .. 128256:
+//  - the CUDA-core GEMV has the least fixed cost and keeps up with the stream for one draft row: M = 1 always,
+//    and M <= 2 (M <= 4) while the weights are under 80 MB (40 MB), where fixed cost decides;
+//  - the vocabulary-rows-on-lanes tensor-core kernel for every other M <= 16 whose h fits in shared memory;
+//  - the draft-rows-on-lanes tensor-core kernel for the rest.
 constexpr int kAutoSmallMaxM = 16;
-constexpr int kAutoGemvMaxM = 2;
+static bool auto_prefers_gemv(int M, int d, int Vt) {
+    if (!gemv_supports(d)) return false;
+    const size_t w_bytes = (size_t)Vt * d * 2;
+    return M == 1 || (M <= 2 && w_bytes <= ((size_t)80 << 20)) || (M <= 4 && w_bytes <= ((size_t)40 << 20));
+}
 
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
     int grid = 0;
@@ -86,10 +93,10 @@ static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
         r = launch_head_mma_small(c, st, &grid);
     } else if (path != VT_PATH_AUTO) {
         return VT_ERR_SHAPE;
+    } else if (auto_prefers_gemv(c.M, c.d, c.Vt)) {
+        r = launch_head_gemv(c, st, &grid);
     } else if (c.M <= kAutoSmallMaxM && (r = launch_head_mma_small(c, st, &grid)) != VT_ERR_UNSUPPORTED) {
         // launched (or failed for a reason another path would not cure)
-    } else if (c.M <= kAutoGemvMaxM && gemv_supports(c.d)) {
-        r = launch_head_gemv(c, st, &grid);
     } else {
         r = launch_head_mma(c, st, &grid);
         if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st, &grid);
