@@ -44,10 +44,11 @@ def head_bytes(d, Vt, M, k):
 
 
 # DRAM traffic of one head launch on the bench workload from the ncu capture summarised in
-# profiles/head_mma_d4096_vt32000_m8.md (dram__bytes_read.sum + dram__bytes_write.sum), valid while the
+# profiles/head_mma_small_d4096_vt32000_m8.md (dram__bytes_read.sum + dram__bytes_write.sum), valid while the
 # kernel sources still hash to the value recorded there.
-NCU_TRAFFIC = {"bytes": 271_346_688 + 3_662_848, "source_hash": "9050caa4aa8c15a1",
-               "sources": ("paper_2603_05210_b200/csrc/vt_head_mma.cu", "paper_2603_05210_b200/csrc/vt_common.cuh")}
+NCU_TRAFFIC = {"bytes": 264_375_808 + 3_532_544, "source_hash": "1a1213be2ec0b1fe",
+               "sources": ("paper_2603_05210_b200/csrc/vt_head_mma_small.cu", "paper_2603_05210_b200/csrc/vt_common.cuh",
+                           "paper_2603_05210_b200/csrc/vt_tc.cuh")}
 
 
 def ncu_traffic_or_none():
@@ -210,6 +211,8 @@ def run_ours(args):
 
     w = WORKLOAD
     d, V, Vt, M, k = w["d"], w["V_full"], w["V_trim"], w["M"], w["k"]
+    if args.m is not None:      # another draft-row count on the same weights (profiling the other head kernels)
+        M = args.m
     tokens = inputs.zipf_token_stream(V, 1.1, 1_000_000, w["seed"])
     ranking = inputs.frequency_ranking(tokens, V)
     case = inputs.make_case("bench", d, Vt, M, k, w["seed"], row_scale=(0.5, 2.0), ranking=ranking)
@@ -283,7 +286,7 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 6), "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAME, "cold": f"calls rotate over {nc} copies of W_trim "
+        "config": {"workload": WORKLOAD_NAME if args.m is None else WORKLOAD_NAME.replace("M=8", f"M={M}"), "cold": f"calls rotate over {nc} copies of W_trim "
                    f"({nc * W_trim.numel() * 2 / 1e6:.0f} MB >= 4x L2 of {l2 / 1e6:.0f} MB): inputs larger than L2",
                    "step": "one vt_draft_head call (contraction + top-k + log-softmax + remap, one launch)",
                    "launch": "eager calls through the binding" if args.no_graph or args.steps < GRAPH_CALLS
@@ -291,7 +294,7 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "calls_per_s": round(1e6 / value, 1)},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
-                     "frac": round(achieved / peak_gbs, 4), "of": peak_kind, "traffic": ncu_traffic_or_none(),
+                     "frac": round(achieved / peak_gbs, 4), "of": peak_kind, "traffic": None if args.m is not None else ncu_traffic_or_none(),
                      "algorithmic_bytes_per_launch": bytes_call, "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
                      "kernel": "head kernel of the chosen path; duration = timed region / launches"},
         "clocks": clocks,
@@ -408,6 +411,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-curve", action="store_true")
+    ap.add_argument("--m", type=int, default=None, help="draft rows M instead of the workload's 8 (not the headline)")
     ap.add_argument("--no-graph", action="store_true", help="launch every timed call through the binding instead of a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
