@@ -75,7 +75,7 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
 //    and M <= 2 (M <= 4) while the weights are under 80 MB (40 MB), where fixed cost decides;
 //  - the vocabulary-rows-on-lanes tensor-core kernel for every other M <= 16 whose h fits in shared memory;
 //  - the draft-rows-on-lanes tensor-core kernel for the rest.
-constexpr int kAutoSmallMaxM = 16;
+constexpr int kAutoSmallMaxM = 64;
 static bool auto_prefers_gemv(int M, int d, int Vt) {
     if (!gemv_supports(d)) return false;
     const size_t w_bytes = (size_t)Vt * d * 2;
@@ -85,24 +85,26 @@ static bool auto_prefers_gemv(int M, int d, int Vt) {
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
     int grid = 0;
     vt_status r;
+    bool merged = c.out.fused_merge != 0;     // the vocabulary-rows-on-lanes kernel always merges row by row itself
     if (path == VT_PATH_GEMV) {
         r = launch_head_gemv(c, st, &grid);
     } else if (path == VT_PATH_MMA) {
         r = launch_head_mma(c, st, &grid);
     } else if (path == VT_PATH_MMA_SMALL) {
         r = launch_head_mma_small(c, st, &grid);
+        merged = true;
     } else if (path != VT_PATH_AUTO) {
         return VT_ERR_SHAPE;
     } else if (auto_prefers_gemv(c.M, c.d, c.Vt)) {
         r = launch_head_gemv(c, st, &grid);
     } else if (c.M <= kAutoSmallMaxM && (r = launch_head_mma_small(c, st, &grid)) != VT_ERR_UNSUPPORTED) {
-        // launched (or failed for a reason another path would not cure)
+        merged = true;     // launched (or failed for a reason another path would not cure)
     } else {
         r = launch_head_mma(c, st, &grid);
         if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st, &grid);
     }
     if (r != VT_OK) return r;
-    if (!c.out.fused_merge) r = launch_merge(c.out, grid, st);
+    if (!merged) r = launch_merge(c.out, grid, st);
     return r;
 }
 

@@ -12,7 +12,7 @@ namespace vt {
 
 // ------------------------------------------------------------------------------------------
 // Workspace of a draft-head call:
-//   [0, 256)                          WsHeader
+//   [0, 512)                          WsHeader
 //   recs [kMaxParts][pitch] u64       per-CTA partial results: M records of KS slots, then padding
 //                                     slots 0..k-1  top-k list as sortable keys, descending, 0-padded
 //                                     slot  k       (running max, sum of exp(x - max)) as two floats
@@ -22,17 +22,17 @@ namespace vt {
 //                                     lanes (one CTA each) with at most 2-way bank conflicts
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxParts = 256;             // upper bound on CTAs that contribute partials
-constexpr size_t kHeaderBytes = 256;
+constexpr size_t kHeaderBytes = 512;
 
-constexpr int kRowTickets = 16;            // draft rows that can be merged row by row (one ticket each)
+constexpr int kRowTickets = 64;            // draft rows that can be merged row by row (one ticket each)
 
 struct WsHeader {
     unsigned int ticket;     // CTAs that have published their partials in the running call
     unsigned int status;     // bit 0: a bounded wait ran out
     unsigned int row_ticket[kRowTickets];   // per draft row: CTAs that have published that row (row-wise merge)
-    unsigned int pad[62 - kRowTickets];
+    unsigned int pad[126 - kRowTickets];
 };
-static_assert(sizeof(WsHeader) == kHeaderBytes, "header is one 256-byte line");
+static_assert(sizeof(WsHeader) == kHeaderBytes, "header is two 256-byte lines");
 
 constexpr unsigned int kStatusTimeout = 1u;
 

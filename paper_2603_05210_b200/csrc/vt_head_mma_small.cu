@@ -1,21 +1,25 @@
-// Draft head, tensor-core path for few draft rows (M <= 16): vocabulary rows on the TMEM lanes.
+// Draft head, tensor-core path for few draft rows (M <= 64): vocabulary rows on the TMEM lanes.
 //
 //   D[i, m] = sum_j W_trim[row0 + i, j] * h[m, j]       (the d -> k linear head, 2*d*k FLOPs per draft row)
 //
-// Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (16 rows: the
-// draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes x 16 columns in tensor
-// memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
+// Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (N = 16, 32, 48 or
+// 64 rows: the draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes x N columns in
+// tensor memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
 // row, so reading a tile out costs one instruction per thread whatever M is, and a weight tile needs no
 // padding rows: the tile height is the CTA's row count split evenly (<= 128), rows of the MMA past it compute
-// on stale shared memory and land in lanes nobody reads.  h stays in shared memory for the whole kernel.
-//   warp 8     TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
-//   warp 9     MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
+// on stale shared memory and land in lanes nobody reads.  For M <= 8 h stays in shared memory for the whole
+// kernel (64 KB at d = 4096); for more draft rows each k-block of h rides in the ring next to its weights (it comes
+// from L2: every CTA reads the same h).
+//   warp 16    TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
+//   warp 17    MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
 //              ring stage; two accumulator buffers in TMEM
 //   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory
-//   warps 0-7  warp w owns draft rows w and w+8: running (max, sum-exp) and top-k of the row over the tile
+//   warps 0-7  (0-15 when M > 8) warp w owns draft rows w, w + 8 (16), ...: running (max, sum-exp) and top-k of the row over the tile
 //              (warp_topk_update), and at the end the row's record, its arrival ticket and, for the warp that
 //              arrives last of all CTAs, the row's final merge (merge_row_global).  No CTA-wide barrier and no
-//              CTA ever waits for another.
+//              CTA ever waits for another.  With more than 16 draft rows a warp owns several, and merging them one
+//              after the other would put several round trips to L2 per row on the critical path: the kernel then
+//              only writes the records and a one-warp-per-row merge kernel follows it.
 // The weight stream is the bound (arithmetic intensity = M FLOP/B).
 #include <cuda.h>
 
@@ -25,27 +29,33 @@
 
 namespace vt {
 
-constexpr int kSmThreads = 320;
-constexpr int kSmEpiWarps = 8;                // warps 0-7; warps 0-3 also read TMEM
-constexpr int kSmProducerWarp = 8, kSmMmaWarp = 9;
-constexpr int kSmMaxM = 16;                   // draft rows = MMA N
+constexpr int kSmMaxEpiWarps = 16;            // warps 0-7, or 0-15 when there are more than 8 draft rows; 0-3 also read TMEM
+constexpr int kSmProducerWarp = kSmMaxEpiWarps, kSmMmaWarp = kSmMaxEpiWarps + 1;
+constexpr int kSmThreads = (kSmMaxEpiWarps + 2) * 32;
+constexpr int kSmMaxM = 64;                   // draft rows <= MMA N <= 64
 constexpr int kSmMaxStages = 32;
 constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
 constexpr int kHParts = 4;                    // h arrives in this many parts so the first MMAs need not wait for all of it
 constexpr int kSmCand = 128 + VT_MAX_K;       // candidate keys per epilogue warp (one tile's columns + the list)
-constexpr uint32_t kSmScratch = kSmCand * 8;
 
 struct SmallParams {
     HeadOut out;
     int M;                    // draft rows, <= kSmMaxM
+    int merge_in_kernel;      // 1: one draft row per epilogue warp, merged by the last warp to publish it; 0: a merge kernel follows
+    int n_epi;                // epilogue warps that take part: 8, or 16 when M > 8 (the rest only meet the final barrier)
+    uint32_t scratch_stride;  // bytes of one epilogue warp's candidate buffer: (128 + k) keys
+    int N;                    // MMA N: M rounded up to a multiple of 16
+    int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
+    uint32_t tmem_cols;       // allocation: 2 accumulators of N columns, a power of two >= 32
     int d, nk;                // nk = 64-column k-blocks
     int TH;                   // vocabulary rows per tile (<= 128)
     int kb_per_stage;         // k-blocks one ring stage holds
     int n_stages;
     uint32_t slot_bytes;      // one k-block of a tile in the ring: TH rounded up to whole 8-row groups x 128 B
+    uint32_t blk_bytes;       // slot_bytes, plus h_blk when h rides in the ring (the h block follows the weights)
     uint32_t stage_bytes;
     uint32_t w_tx;            // bytes one W box delivers (TH * 128)
-    uint32_t h_blk;           // bytes of one k-block of h: 8 or 16 rows x 128 B
+    uint32_t h_blk;           // bytes of one k-block of h: 8 rows (M <= 8) or N rows x 128 B
     uint32_t h_off, lg_off, list_off, scratch_off, bar_off, total_smem;   // from the 1024-aligned base
     uint32_t idesc;
 };
@@ -59,7 +69,7 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "r"(taddr) : "memory");
 }
 // Barrier among the epilogue warps only (the producer and the MMA issuer never join it).
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kSmEpiWarps * 32) : "memory"); }
+__device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); }
 
 __global__ void __launch_bounds__(kSmThreads, 1)
 head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
@@ -81,7 +91,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     float* lg = reinterpret_cast<float*>(smem + p.lg_off);                                  // [M][kLgPitch]
     unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [M][k]
     float2* ms_s = reinterpret_cast<float2*>(lists + (size_t)M * k);                         // [kSmMaxM]
-    unsigned char* scratch = smem + p.scratch_off + (uint32_t)(warp & 7) * kSmScratch;
+    float* tau_s = reinterpret_cast<float*>(ms_s + kSmMaxM);                                 // [kSmMaxM] k-th best logit so far
+    unsigned char* scratch = smem + p.scratch_off + (uint32_t)(warp & (kSmMaxEpiWarps - 1)) * p.scratch_stride;
     const uint32_t bar_full = base + p.bar_off, bar_empty = bar_full + 8u * S;
     const uint32_t bar_accf = bar_empty + 8u * S, bar_acce = bar_accf + 16u;
     const uint32_t bar_h = bar_acce + 16u, bar_drain = bar_h + 8u * kHParts;
@@ -107,13 +118,19 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         fence_mbar_init();
     }
     for (int i = tid; i < M * k; i += blockDim.x) lists[i] = 0ull;
-    if (tid < kSmMaxM) ms_s[tid] = make_float2(-INFINITY, 0.0f);
-    // With 8 rows of h per k-block the MMA's rows 8-15 alias the next k-block; the last one reads this pad.
-    for (int i = tid; i < 256; i += blockDim.x)
-        reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
+    if (tid < kSmMaxM) {
+        ms_s[tid] = make_float2(-INFINITY, 0.0f);
+        tau_s[tid] = -INFINITY;
+    }
+    // With 8 rows of h per k-block the MMA's rows 8-15 alias whatever follows the block (the next k-block of a
+    // resident h, the next ring slot otherwise): accumulator columns nobody reads.  After the last block of a
+    // resident h that is this pad.
+    if (p.h_resident)
+        for (int i = tid; i < 256; i += blockDim.x)
+            reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
     if (warp == kSmMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"(32u) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     fence_proxy_async();          // the zeroed pad is read by the tensor core (async proxy)
@@ -147,10 +164,12 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (*abort_flag) { ok = false; break; }
                     const int nb = min(kbs, nk - ks);
                     const uint32_t bar = bar_full + 8u * s;
-                    mbar_arrive_expect_tx(bar, (uint32_t)nb * p.w_tx);
-                    for (int kb = 0; kb < nb; ++kb)
-                        tma_load_2d_hint(base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.slot_bytes, &tmW,
-                                         (ks + kb) * kBoxK, row0, bar, stream_once);
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (p.w_tx + (p.h_resident ? 0u : p.h_blk)));
+                    for (int kb = 0; kb < nb; ++kb) {
+                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
+                        tma_load_2d_hint(dst, &tmW, (ks + kb) * kBoxK, row0, bar, stream_once);
+                        if (!p.h_resident) tma_load_2d(dst + p.slot_bytes, &tmH, (ks + kb) * kBoxK, 0, bar);
+                    }
                     ++issued;
                     if (++s == S) { s = 0; ++wrap; }
                 }
@@ -169,16 +188,17 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             const uint64_t desc0 = smem_desc_sw128(base);                      // descriptor of the ring's first byte
             const uint64_t h_desc0 = smem_desc_sw128(base + p.h_off);
             const uint32_t stage_units = p.stage_bytes >> 4, slot_units = p.slot_bytes >> 4, h_units = p.h_blk >> 4;
+            const uint32_t blk_units = p.blk_bytes >> 4;
             const int kbs = p.kb_per_stage;
             int h_ready = 0;                                                   // k-blocks of h known to have landed
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 16);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.N);
                 for (int ks = 0; ks < nk && ok; ks += kbs) {
                     const int nb = min(kbs, nk - ks);
-                    while (h_ready < ks + nb) {
+                    while (p.h_resident && h_ready < ks + nb) {
                         if (!mbar_wait(bar_h + 8u * (uint32_t)(h_ready / h_part), 0u)) { fail(); ok = false; break; }
                         h_ready += h_part;
                     }
@@ -187,8 +207,9 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (*abort_flag) { ok = false; break; }
                     tc_fence_after();
                     for (int kb = 0; kb < nb; ++kb) {
-                        const uint64_t a_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * slot_units);
-                        const uint64_t b_desc = h_desc0 + (uint64_t)((uint32_t)(ks + kb) * h_units);
+                        const uint64_t a_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * blk_units);
+                        const uint64_t b_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)(ks + kb) * h_units)
+                                                             : a_desc + slot_units;
                         // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
                         tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
                         tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
@@ -205,9 +226,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 (void)mbar_wait(bar_drain, 0u);
             }
         }
-    } else {
-        // ------------------------------------------------------------------ epilogue warps 0-7
-        if (warp == kSmEpiWarps - 1 && lane == 0 && ntiles > 0) {
+    } else if (warp < p.n_epi) {
+        // ------------------------------------------------------------------ epilogue warps
+        const int n_epi = p.n_epi;
+        if (warp == n_epi - 1 && lane == 0 && ntiles > 0 && p.h_resident) {
             // h, fetched once: every CTA needs all of it, one box per k-block, in kHParts parts
             for (int j = 0; j < kHParts; ++j) {
                 const int k0 = j * h_part, k1 = min(nk, k0 + h_part);
@@ -219,7 +241,6 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         }
         __syncwarp();
         unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(scratch);
-        float tau[2] = {-INFINITY, -INFINITY};
         // Every epilogue warp passes the same two barriers per tile whatever happens, so none can be left
         // waiting at one: after a wait has run out the remaining tiles only skip their work.
         for (int t = 0; t < ntiles; ++t) {
@@ -235,45 +256,49 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 }
                 if (got) {
                     tc_fence_after();
-                    uint32_t r[16];
-                    tc_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 16), r);
-                    tc_wait_ld();
+                    const int i = warp * 32 + lane;                    // TMEM lane = vocabulary row of the tile
+                    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
+                    for (int c0 = 0; c0 < p.N; c0 += 16) {             // 16 draft rows at a time
+                        uint32_t r[16];
+                        tc_ld16(taddr + (uint32_t)c0, r);
+                        tc_wait_ld();
+                        if (i < nv) {
+#pragma unroll
+                            for (int m = 0; m < 16; ++m)
+                                if (c0 + m < M) lg[(c0 + m) * kLgPitch + i] = __uint_as_float(r[m]);
+                            if (p.out.logits) {
+#pragma unroll
+                                for (int m = 0; m < 16; ++m)
+                                    if (c0 + m < M) p.out.logits[(size_t)(c0 + m) * Vt + row0 + i] = __uint_as_float(r[m]);
+                            }
+                        }
+                    }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
-                    const int i = warp * 32 + lane;                    // TMEM lane = vocabulary row of the tile
-                    if (i < nv) {
-#pragma unroll
-                        for (int m = 0; m < kSmMaxM; ++m)
-                            if (m < M) lg[m * kLgPitch + i] = __uint_as_float(r[m]);
-                        if (p.out.logits) {
-#pragma unroll
-                            for (int m = 0; m < kSmMaxM; ++m)
-                                if (m < M) p.out.logits[(size_t)m * Vt + row0 + i] = __uint_as_float(r[m]);
-                        }
-                    }
                 }
             }
-            epi_barrier();                                             // the tile's logits are in shared memory
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int m = warp + kSmEpiWarps * q;
-                if (m < M)
-                    tau[q] = warp_topk_update<4>(lg + m * kLgPitch, nv, row0, lists + (size_t)m * k, k, tau[q], cbuf,
-                                                 ms_s + m, lane);
+            epi_barrier(n_epi * 32);                                   // the tile's logits are in shared memory
+            for (int m = warp; m < M; m += n_epi) {
+                const float tau = warp_topk_update<4>(lg + m * kLgPitch, nv, row0, lists + (size_t)m * k, k, tau_s[m], cbuf,
+                                                      ms_s + m, lane);
+                __syncwarp();
+                if (lane == 0) tau_s[m] = tau;
+                __syncwarp();
             }
-            epi_barrier();                                             // ... and may be overwritten
+            epi_barrier(n_epi * 32);                                   // ... and may be overwritten
         }
         // ------------------------------------------------------------------ publish, and merge if last
         // The warp owns its rows from the first tile to the outputs: record -> fence -> ticket; the warp that
         // draws the last ticket of a row (over all CTAs) merges that row.  No CTA-wide step in between.
-        for (int m = warp; m < M; m += kSmEpiWarps) {
+        for (int m = warp; m < M; m += n_epi) {
             const unsigned long long* list = lists + (size_t)m * k;
             for (int j = lane; j < k; j += 32) VT_ROW_KEYS(p.out, m, j)[cta] = list[j];
             if (lane == 0) {
                 const float2 ms = ms_s[m];
                 VT_ROW_MS(p.out, m)[cta] = pack_ms(ms.x, ms.y);
             }
+            if (!p.merge_in_kernel) continue;      // the records are complete when the kernel is
             __threadfence();
             __syncwarp();
             unsigned int ticket = 0;
@@ -285,7 +310,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 if (lane == 0) p.out.hdr->row_ticket[m] = 0u;          // ready for the next call
             }
         }
-        if (warp == kSmEpiWarps - 1 && lane == 0 && ntiles > 0 && *abort_flag) {
+        if (warp == n_epi - 1 && lane == 0 && ntiles > 0 && p.h_resident && *abort_flag) {
             // let the copies of h land before the CTA gives its shared memory back
             for (int j = 0; j < kHParts && j * h_part < nk; ++j) (void)mbar_wait(bar_h + 8u * j, 0u);
         }
@@ -295,48 +320,66 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     __syncthreads();
     tc_fence_after();
     if (warp == kSmMmaWarp)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------ host
-// Shared memory the kernel needs beside the ring, and the tile geometry, for a shape; false if h does not fit.
+// Tile geometry and shared-memory layout for a shape; false if it does not fit.
 static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     if (M < 1 || M > kSmMaxM) return false;
     const int R = (Vt + grid - 1) / grid;                    // most rows a CTA owns
     const int nt = (R + 127) / 128;
     p->M = M;
+    p->N = ((M + 15) / 16) * 16;
     p->d = d;
     p->nk = (d + kBoxK - 1) / kBoxK;
     p->TH = (R + nt - 1) / nt;
     p->w_tx = (uint32_t)p->TH * 128u;
     p->slot_bytes = (uint32_t)((p->TH + 7) / 8) * 1024u;
-    p->h_blk = M <= 8 ? 1024u : 2048u;
-    // a stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height
-    p->kb_per_stage = std::max(1, std::min(std::min(4, p->nk), (int)((28 * 1024 + p->slot_bytes / 2) / p->slot_bytes)));
-    p->stage_bytes = p->slot_bytes * (uint32_t)p->kb_per_stage;
-    // instruction descriptor: D fp32, A and B bf16, both K-major, N = 16, M = 128
-    p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-    const size_t h_bytes = (size_t)p->nk * p->h_blk + 1024;               // + the pad the last k-block's rows 8-15 read
-    const size_t lg_bytes = (size_t)M * kLgPitch * 4;
-    const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 8) + 127) & ~(size_t)127;
-    const size_t scratch_bytes = ((size_t)kSmEpiWarps * kSmScratch + 127) & ~(size_t)127;
+    p->h_blk = M <= 8 ? 1024u : (uint32_t)p->N * 128u;
+    p->tmem_cols = 32;
+    while (p->tmem_cols < 2u * (uint32_t)p->N) p->tmem_cols *= 2;
+    // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 128
+    p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const size_t lg_bytes = ((size_t)M * kLgPitch * 4 + 127) & ~(size_t)127;
+    const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
+    p->n_epi = M > 8 ? kSmMaxEpiWarps : 8;
+    p->merge_in_kernel = M <= p->n_epi;
+    p->scratch_stride = (uint32_t)(kSmCand - VT_MAX_K + k) * 8u;
+    const size_t scratch_bytes = ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
     const size_t bar_bytes = (size_t)(2 * kSmMaxStages + 4 + kHParts + 1) * 8 + 16;
-    const size_t fixed = 1024 + h_bytes + ((lg_bytes + 127) & ~(size_t)127) + list_bytes + scratch_bytes + bar_bytes + 128;
-    if (fixed + 2 * (size_t)p->stage_bytes > (size_t)kMaxDynSmem) return false;
-    const int S = (int)std::min<size_t>(kSmMaxStages, ((size_t)kMaxDynSmem - fixed) / p->stage_bytes);
-    const size_t ring = (size_t)S * p->stage_bytes;
-    if (S < 3) return false;                                              // too few bytes in flight to be worth it
-    p->n_stages = S;
-    p->h_off = (uint32_t)ring;                                            // stages are multiples of 1024 bytes
-    p->lg_off = (uint32_t)(ring + h_bytes);
-    p->list_off = (uint32_t)(p->lg_off + ((lg_bytes + 127) & ~(size_t)127));
-    p->scratch_off = (uint32_t)(p->list_off + list_bytes);
-    p->bar_off = (uint32_t)(p->scratch_off + scratch_bytes);
-    // An MMA always reads 128 A rows = 16 KB from its slot's first byte: past a short tile that is whatever
-    // follows in shared memory, which must still be inside the allocation.
-    const size_t need = std::max((size_t)p->bar_off + bar_bytes, ring - p->slot_bytes + 16384);
-    p->total_smem = (uint32_t)(need + 1024);
-    return p->total_smem <= (uint32_t)kMaxDynSmem;
+    const size_t common = 1024 + lg_bytes + list_bytes + scratch_bytes + bar_bytes + 128;
+    // h resident (M <= 8 only: 8 rows per k-block) when that still leaves a ring of four stages; else it streams
+    for (int attempt = M <= 8 ? 0 : 1; attempt < 3; ++attempt) {
+        const int resident = attempt == 0;
+        const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 : 0;    // + the pad the last block's rows 8-15 read
+        p->h_resident = resident;
+        p->blk_bytes = p->slot_bytes + (resident ? 0u : p->h_blk);
+        // A stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height; two k-blocks at
+        // least (four MMAs per hand-over are too few), one only as the last resort.
+        p->kb_per_stage = std::max(2, std::min(4, (int)((28 * 1024 + p->blk_bytes / 2) / p->blk_bytes)));
+        if (attempt == 2) p->kb_per_stage = 1;
+        p->kb_per_stage = std::min(p->kb_per_stage, p->nk);
+        p->stage_bytes = p->blk_bytes * (uint32_t)p->kb_per_stage;
+        const size_t fixed = common + h_bytes;
+        if (fixed + 3 * (size_t)p->stage_bytes > (size_t)kMaxDynSmem) continue;
+        const int S = (int)std::min<size_t>(kSmMaxStages, ((size_t)kMaxDynSmem - fixed) / p->stage_bytes);
+        if (S < (resident ? 4 : 3)) continue;
+        const size_t ring = (size_t)S * p->stage_bytes;
+        p->n_stages = S;
+        p->h_off = (uint32_t)ring;                                            // stages are multiples of 1024 bytes
+        p->lg_off = (uint32_t)(ring + h_bytes);
+        p->list_off = (uint32_t)(p->lg_off + lg_bytes);
+        p->scratch_off = (uint32_t)(p->list_off + list_bytes);
+        p->bar_off = (uint32_t)(p->scratch_off + scratch_bytes);
+        // An MMA always reads 128 A rows = 16 KB from its slot's first byte and N B rows from its h block's: past
+        // a short tile or an 8-row h block that is whatever follows in shared memory, which must still be inside
+        // the allocation.
+        const size_t need = std::max((size_t)p->bar_off + bar_bytes, ring + 16384);
+        p->total_smem = (uint32_t)(need + 1024);
+        if (p->total_smem <= (uint32_t)kMaxDynSmem) return true;
+    }
+    return false;
 }
 
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_out) {
@@ -346,7 +389,7 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
     SmallParams p{};
-    if (!c.out.fused_merge || !small_plan(c.M, c.d, c.Vt, c.out.k, grid, &p)) return VT_ERR_UNSUPPORTED;
+    if (!small_plan(c.M, c.d, c.Vt, c.out.k, grid, &p)) return VT_ERR_UNSUPPORTED;
     p.out = c.out;
 
     static int configured_device = -1;
@@ -365,7 +408,8 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     cudaError_t e = launch_pdl(head_mma_small_kernel, grid, kSmThreads, p.total_smem, st, tmW, tmH, p);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
-    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return p.merge_in_kernel ? VT_OK : launch_merge_rowmajor(c.out, grid, st);
 }
 
 }  // namespace vt
