@@ -10,8 +10,8 @@
 // on stale shared memory and land in lanes nobody reads.  For M <= 8 h stays in shared memory for the whole
 // kernel (64 KB at d = 4096); for more draft rows each k-block of h rides in the ring next to its weights (it comes
 // from L2: every CTA reads the same h).
-//   warp 16    TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
-//   warp 17    MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
+//   next warp  TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
+//   last warp  MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
 //              ring stage; two accumulator buffers in TMEM
 //   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory
 //   warps 0-7  (0-15 when M > 8) warp w owns draft rows w, w + 8 (16), ...: running (max, sum-exp) and top-k of the row over the tile
@@ -30,8 +30,7 @@
 namespace vt {
 
 constexpr int kSmMaxEpiWarps = 16;            // warps 0-7, or 0-15 when there are more than 8 draft rows; 0-3 also read TMEM
-constexpr int kSmProducerWarp = kSmMaxEpiWarps, kSmMmaWarp = kSmMaxEpiWarps + 1;
-constexpr int kSmThreads = (kSmMaxEpiWarps + 2) * 32;
+constexpr int kSmThreads = (kSmMaxEpiWarps + 2) * 32;     // at most: the epilogue warps, then the producer, then the MMA issuer
 constexpr int kSmMaxM = 64;                   // draft rows <= MMA N <= 64
 constexpr int kSmMaxStages = 32;
 constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
@@ -42,7 +41,7 @@ struct SmallParams {
     HeadOut out;
     int M;                    // draft rows, <= kSmMaxM
     int merge_in_kernel;      // 1: one draft row per epilogue warp, merged by the last warp to publish it; 0: a merge kernel follows
-    int n_epi;                // epilogue warps that take part: 8, or 16 when M > 8 (the rest only meet the final barrier)
+    int n_epi;                // epilogue warps: 8, or 16 when M > 8; the block has two more (producer, MMA issuer)
     uint32_t scratch_stride;  // bytes of one epilogue warp's candidate buffer: (128 + k) keys
     int N;                    // MMA N: M rounded up to a multiple of 16
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
@@ -80,6 +79,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     unsigned char* smem = smem_raw + (base - raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int producer_warp = p.n_epi, mma_warp = p.n_epi + 1;     // the block has n_epi + 2 warps
     const int G = gridDim.x, cta = blockIdx.x;
     const int Vt = p.out.Vt, k = p.out.k, M = p.M, TH = p.TH, S = p.n_stages, nk = p.nk;
     const int row_begin = (int)((long long)cta * Vt / G);
@@ -99,7 +99,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + p.bar_off + 8u * (2 * S + 4 + kHParts + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    if (warp == kSmProducerWarp && lane == 0) {      // descriptor fetches overlap the barrier set-up below
+    if (warp == producer_warp && lane == 0) {      // descriptor fetches overlap the barrier set-up below
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
     }
@@ -128,7 +128,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     if (p.h_resident)
         for (int i = tid; i < 256; i += blockDim.x)
             reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
-    if (warp == kSmMmaWarp) {
+    if (warp == mma_warp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -149,7 +149,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         atomicOr(&p.out.hdr->status, kStatusTimeout);
     };
 
-    if (warp == kSmProducerWarp) {
+    if (warp == producer_warp) {
         // ------------------------------------------------------------------ TMA producer: the weight stream
         if (lane == 0) {
             int s = 0, issued = 0;
@@ -179,7 +179,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     (void)mbar_wait(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u);
             }
         }
-    } else if (warp == kSmMmaWarp) {
+    } else if (warp == mma_warp) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             int s = 0;
@@ -319,7 +319,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == kSmMmaWarp)
+    if (warp == mma_warp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
 }
 
@@ -405,7 +405,7 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     if (r != VT_OK) return r;
     r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
     if (r != VT_OK) return r;
-    cudaError_t e = launch_pdl(head_mma_small_kernel, grid, kSmThreads, p.total_smem, st, tmW, tmH, p);
+    cudaError_t e = launch_pdl(head_mma_small_kernel, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e);
