@@ -72,14 +72,14 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
 
 // Automatic path choice, from measurements at d = 4096 over V_trim = 4096 .. 128256:
 //  - the CUDA-core GEMV has the least fixed cost and keeps up with the stream for one draft row: M = 1 always,
-//    and M <= 2 (M <= 4) while the weights are under 80 MB (40 MB), where fixed cost decides;
-//  - the vocabulary-rows-on-lanes tensor-core kernel for every other M <= 16 whose h fits in shared memory;
+//    and M = 2 while the weights are under 80 MB, where fixed cost decides;
+//  - the vocabulary-rows-on-lanes tensor-core kernel for every other M <= 64;
 //  - the draft-rows-on-lanes tensor-core kernel for the rest.
 constexpr int kAutoSmallMaxM = 64;
 static bool auto_prefers_gemv(int M, int d, int Vt) {
     if (!gemv_supports(d)) return false;
     const size_t w_bytes = (size_t)Vt * d * 2;
-    return M == 1 || (M <= 2 && w_bytes <= ((size_t)80 << 20)) || (M <= 4 && w_bytes <= ((size_t)40 << 20));
+    return M == 1 || (M == 2 && w_bytes <= ((size_t)80 << 20));
 }
 
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {

@@ -20,6 +20,13 @@
 //              CTA ever waits for another.  With more than 16 draft rows a warp owns several, and merging them one
 //              after the other would put several round trips to L2 per row on the critical path: the kernel then
 //              only writes the records and a one-warp-per-row merge kernel follows it.
+// Short tiles (a CTA with at most 64 rows: V_trim up to about 9,500) would waste the MMA: it costs the same 60-80
+// cycles for 28 live rows as for 128, and 4 * nk of them per tile is then what the call takes.  With M <= 8 the
+// kernel folds G = 4 (2) k-blocks into one MMA instead: TMEM lanes 32g..32g+31 (64g..) hold the tile's rows for
+// k-block G*j + g, and since an 8-row block of h per k-block is already laid out 1 KB after the other, a B
+// operand of N = 8 * G rows is the matching k-blocks of h.  Lane group g against column group g is the wanted
+// partial sum (the other G - 1 column groups are cross terms nobody reads); the readers add the G partial sums
+// through shared memory.  G times fewer MMAs per tile.
 // The weight stream is the bound (arithmetic intensity = M FLOP/B).
 #include <cuda.h>
 
@@ -47,10 +54,14 @@ struct SmallParams {
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
     uint32_t tmem_cols;       // allocation: 2 accumulators of N columns, a power of two >= 32
     int d, nk;                // nk = 64-column k-blocks
+    int G;                    // k-blocks folded into one MMA: 128 / (tile height rounded up to 32 or 64), M <= 8 only, else 1
+    int nsb;                  // MMA steps along d: ceil(nk / G) "super-blocks" of G k-blocks
     int TH;                   // vocabulary rows per tile (<= 128)
     int kb_per_stage;         // k-blocks one ring stage holds
     int n_stages;
     uint32_t slot_bytes;      // one k-block of a tile in the ring: TH rounded up to whole 8-row groups x 128 B
+    uint32_t sub_bytes;       // with folded k-blocks: bytes between the k-blocks of one MMA step in a slot (128 / G rows x 128 B)
+    uint32_t part_off;        // with folded k-blocks: the readers' partial sums [G][8][64] floats
     uint32_t blk_bytes;       // slot_bytes, plus h_blk when h rides in the ring (the h block follows the weights)
     uint32_t stage_bytes;
     uint32_t w_tx;            // bytes one W box delivers (TH * 128)
@@ -67,6 +78,14 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr) : "memory");
+}
+// Barrier among the four TMEM-reading warps.
+__device__ __forceinline__ void reader_barrier() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 // Barrier among the epilogue warps only (the producer and the MMA issuer never join it).
 __device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); }
 
@@ -81,7 +100,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int producer_warp = p.n_epi, mma_warp = p.n_epi + 1;     // the block has n_epi + 2 warps
     const int G = gridDim.x, cta = blockIdx.x;
-    const int Vt = p.out.Vt, k = p.out.k, M = p.M, TH = p.TH, S = p.n_stages, nk = p.nk;
+    const int Vt = p.out.Vt, k = p.out.k, M = p.M, TH = p.TH, S = p.n_stages, nk = p.nk, KF = p.G, nsb = p.nsb;   // KF: k-blocks folded into one MMA
     const int row_begin = (int)((long long)cta * Vt / G);
     const int row_end = (int)((long long)(cta + 1) * Vt / G);
     const int nrows = row_end - row_begin;
@@ -125,8 +144,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     // With 8 rows of h per k-block the MMA's rows 8-15 alias whatever follows the block (the next k-block of a
     // resident h, the next ring slot otherwise): accumulator columns nobody reads.  After the last block of a
     // resident h that is this pad.
+    // With folded k-blocks the last MMA step may name k-blocks past d: zeros here, zeros (out-of-range boxes)
+    // from the TMA on the weight side.
     if (p.h_resident)
-        for (int i = tid; i < 256; i += blockDim.x)
+        for (int i = tid; i < 256 * KF; i += blockDim.x)
             reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
     if (warp == mma_warp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -159,15 +180,18 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             const uint64_t stream_once = l2_policy_evict_first();
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int row0 = row_begin + t * TH;
-                for (int ks = 0; ks < nk; ks += kbs) {
+                for (int ks = 0; ks < nsb; ks += kbs) {
                     if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
                     if (*abort_flag) { ok = false; break; }
-                    const int nb = min(kbs, nk - ks);
+                    const int nb = min(kbs, nsb - ks);
                     const uint32_t bar = bar_full + 8u * s;
-                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (p.w_tx + (p.h_resident ? 0u : p.h_blk)));
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * ((uint32_t)KF * p.w_tx + (p.h_resident ? 0u : p.h_blk)));
                     for (int kb = 0; kb < nb; ++kb) {
                         const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
-                        tma_load_2d_hint(dst, &tmW, (ks + kb) * kBoxK, row0, bar, stream_once);
+                        // k-block KF * (ks + kb) + g goes to lanes g * (128 / KF) ...; one past d is all zero fill
+                        for (int g = 0; g < KF; ++g)
+                            tma_load_2d_hint(dst + (uint32_t)g * p.sub_bytes, &tmW, ((ks + kb) * KF + g) * kBoxK, row0, bar,
+                                             stream_once);
                         if (!p.h_resident) tma_load_2d(dst + p.slot_bytes, &tmH, (ks + kb) * kBoxK, 0, bar);
                     }
                     ++issued;
@@ -196,9 +220,9 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 if (t >= 2 && !mbar_wait(bar_acce + 8u * buf, (uint32_t)((t >> 1) - 1) & 1u)) { fail(); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.N);
-                for (int ks = 0; ks < nk && ok; ks += kbs) {
-                    const int nb = min(kbs, nk - ks);
-                    while (p.h_resident && h_ready < ks + nb) {
+                for (int ks = 0; ks < nsb && ok; ks += kbs) {
+                    const int nb = min(kbs, nsb - ks);
+                    while (p.h_resident && h_ready < min(nk, (ks + nb) * KF)) {
                         if (!mbar_wait(bar_h + 8u * (uint32_t)(h_ready / h_part), 0u)) { fail(); ok = false; break; }
                         h_ready += h_part;
                     }
@@ -208,7 +232,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     tc_fence_after();
                     for (int kb = 0; kb < nb; ++kb) {
                         const uint64_t a_desc = desc0 + (uint64_t)((uint32_t)s * stage_units + (uint32_t)kb * blk_units);
-                        const uint64_t b_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)(ks + kb) * h_units)
+                        const uint64_t b_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)((ks + kb) * KF) * h_units)
                                                              : a_desc + slot_units;
                         // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
                         tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
@@ -254,10 +278,35 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u));
                     if (!got) fail();
                 }
-                if (got) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
+                if (KF > 1) {
+                    // Folded k-blocks: this warp's lanes are k-group g of tile rows r0 + lane, and columns 8g..8g+7
+                    // of the accumulator are their partial logits for the (up to 8) draft rows.
+                    const int SR = 128 / KF, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
+                    float* part = reinterpret_cast<float*>(smem + p.part_off);
+                    if (got) {
+                        tc_fence_after();
+                        uint32_t v[8];
+                        tc_ld8(taddr + (uint32_t)(8 * g), v);
+                        tc_wait_ld();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+#pragma unroll
+                        for (int m = 0; m < 8; ++m) part[(g * 8 + m) * 64 + r] = __uint_as_float(v[m]);
+                    }
+                    reader_barrier();                                  // all four readers' partial sums are in place
+                    for (int e = tid; e < M * SR; e += 128) {
+                        const int m = e / SR, rr = e - m * SR;
+                        if (rr >= nv) continue;
+                        float sum = 0.0f;
+                        for (int gg = 0; gg < KF; ++gg) sum += part[(gg * 8 + m) * 64 + rr];
+                        lg[m * kLgPitch + rr] = sum;
+                        if (p.out.logits) p.out.logits[(size_t)m * Vt + row0 + rr] = sum;
+                    }
+                } else if (got) {
                     tc_fence_after();
                     const int i = warp * 32 + lane;                    // TMEM lane = vocabulary row of the tile
-                    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
                     for (int c0 = 0; c0 < p.N; c0 += 16) {             // 16 draft rows at a time
                         uint32_t r[16];
                         tc_ld16(taddr + (uint32_t)c0, r);
@@ -330,17 +379,11 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     const int R = (Vt + grid - 1) / grid;                    // most rows a CTA owns
     const int nt = (R + 127) / 128;
     p->M = M;
-    p->N = ((M + 15) / 16) * 16;
     p->d = d;
     p->nk = (d + kBoxK - 1) / kBoxK;
     p->TH = (R + nt - 1) / nt;
     p->w_tx = (uint32_t)p->TH * 128u;
-    p->slot_bytes = (uint32_t)((p->TH + 7) / 8) * 1024u;
-    p->h_blk = M <= 8 ? 1024u : (uint32_t)p->N * 128u;
-    p->tmem_cols = 32;
-    while (p->tmem_cols < 2u * (uint32_t)p->N) p->tmem_cols *= 2;
-    // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 128
-    p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    p->h_blk = M <= 8 ? 1024u : (uint32_t)(((M + 15) / 16) * 16) * 128u;
     const size_t lg_bytes = ((size_t)M * kLgPitch * 4 + 127) & ~(size_t)127;
     const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
     p->n_epi = M > 8 ? kSmMaxEpiWarps : 8;
@@ -352,23 +395,36 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     // h resident (M <= 8 only: 8 rows per k-block) when that still leaves a ring of four stages; else it streams
     for (int attempt = M <= 8 ? 0 : 1; attempt < 3; ++attempt) {
         const int resident = attempt == 0;
-        const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 : 0;    // + the pad the last block's rows 8-15 read
+        // short tiles with a resident 8-row h: fold G k-blocks into each MMA
+        p->G = !resident ? 1 : p->TH <= 32 ? 4 : p->TH <= 64 ? 2 : 1;
+        p->nsb = (p->nk + p->G - 1) / p->G;
+        p->N = p->G > 1 ? 8 * p->G : ((M + 15) / 16) * 16;
+        p->sub_bytes = (uint32_t)(128 / p->G) * 128u;
+        p->slot_bytes = p->G > 1 ? 16384u : (uint32_t)((p->TH + 7) / 8) * 1024u;
+        p->tmem_cols = 32;
+        while (p->tmem_cols < 2u * (uint32_t)p->N) p->tmem_cols *= 2;
+        // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 128
+        p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const size_t part_bytes = p->G > 1 ? (size_t)p->G * 8 * 64 * 4 : 0;
+        // + zeros for what the last MMA step reads past h: rows 8-15 of an unfolded step, whole k-blocks of a folded one
+        const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 * (size_t)p->G : 0;
         p->h_resident = resident;
         p->blk_bytes = p->slot_bytes + (resident ? 0u : p->h_blk);
         // A stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height; two k-blocks at
         // least (four MMAs per hand-over are too few), one only as the last resort.
         p->kb_per_stage = std::max(2, std::min(4, (int)((28 * 1024 + p->blk_bytes / 2) / p->blk_bytes)));
         if (attempt == 2) p->kb_per_stage = 1;
-        p->kb_per_stage = std::min(p->kb_per_stage, p->nk);
+        p->kb_per_stage = std::min(p->kb_per_stage, p->nsb);
         p->stage_bytes = p->blk_bytes * (uint32_t)p->kb_per_stage;
-        const size_t fixed = common + h_bytes;
+        const size_t fixed = common + h_bytes + part_bytes;
         if (fixed + 3 * (size_t)p->stage_bytes > (size_t)kMaxDynSmem) continue;
         const int S = (int)std::min<size_t>(kSmMaxStages, ((size_t)kMaxDynSmem - fixed) / p->stage_bytes);
-        if (S < (resident ? 4 : 3)) continue;
+        if (S < (resident && p->G == 1 ? 4 : 3)) continue;
         const size_t ring = (size_t)S * p->stage_bytes;
         p->n_stages = S;
         p->h_off = (uint32_t)ring;                                            // stages are multiples of 1024 bytes
-        p->lg_off = (uint32_t)(ring + h_bytes);
+        p->part_off = (uint32_t)(ring + h_bytes);
+        p->lg_off = (uint32_t)(p->part_off + part_bytes);
         p->list_off = (uint32_t)(p->lg_off + lg_bytes);
         p->scratch_off = (uint32_t)(p->list_off + list_bytes);
         p->bar_off = (uint32_t)(p->scratch_off + scratch_bytes);

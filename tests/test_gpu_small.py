@@ -210,6 +210,16 @@ def test_all_paths_agree_on_logits(vt):
     assert np.max(np.abs(a - b)) <= 2e-3 and np.max(np.abs(a - c)) <= 2e-3
 
 
+@pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (16, 1), (17, 2), (64, 2), (65, 2), (300, 4)])
+def test_launches_per_call_of_the_automatic_choice(vt, oracle, M, launches):
+    # M = 1: GEMV; M <= 16: one launch, rows merged by the last warp to publish them; M <= 64: the same kernel
+    # followed by the row-wise merge kernel; beyond: the draft-rows-on-lanes kernel in passes of 128 rows, then a merge
+    h, W, d2t = rand_case(M, 256, 3000, seed=40 + M)
+    got = run_head(vt, h, dev_bf16(W), d2t, 4, vt.VT_PATH_AUTO)
+    assert vt.vt_last_launch_count() == launches
+    parity.check_head(got, oracle.draft_head(h, W, d2t, 4, want_logits=True), d2t, 4)
+
+
 def test_forced_small_path_refuses_many_draft_rows(vt):
     h, W, d2t = rand_case(65, 64, 100, seed=12)
     with pytest.raises(vt.VtError) as e:
