@@ -86,17 +86,15 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
     unsigned char* hs = smem + p.h_off;                                                      // [MP][d] bf16
     unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [consumer][NV][KS]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + p.bar_off);
-    // bars: full[S], empty[S], merge; then two ints: abort flag, last flag
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * S, bar_merge = bar_empty + 8u * S;
+    // bars: full[S], empty[S], one spare; then the abort flag
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * S;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * S + 1);
-    int* last_flag = const_cast<int*>(abort_flag) + 1;
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8u * s, 1);
             mbar_init(bar_empty + 8u * s, 1);
         }
-        mbar_init(bar_merge, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -218,17 +216,29 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         const unsigned long long* rec0 = lists + (size_t)m * KS;
         const int stride = MP * KS;
         const float2 ms = warp_merge_ms(rec0, stride, P1, k);
-        unsigned long long* dst = VT_REC(p.out, cta, p.m_begin + m);
         unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(smem + p.fold_off) + (size_t)warp * kMergeCand;
-        warp_select_topk(rec0, stride, P1, k, cbuf, [&](int j, unsigned long long best) { dst[j] = best; });
-        if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
-    }
-
-    // ---------------------------------------------------------------------- publish (+ merge)
-    if (!p.out.fused_merge) return;
-    if (publish_and_check_last(p.out.hdr, last_flag)) {
-        merge_rows(p.out, G, p.m_begin, p.m_count, smem, p.bar_off, bar_merge);   // ring, h and lists are free now
-        if (tid == 0) p.out.hdr->ticket = 0u;                                      // ready for the next call
+        if (p.out.fused_merge) {
+            // Row-major record, then the row's ticket: the warp that draws the last one (over all CTAs) merges the
+            // row at once, straight from global memory.  No CTA-wide step between the fold and the outputs.
+            const int row = p.m_begin + m;
+            warp_select_topk(rec0, stride, P1, k, cbuf,
+                             [&](int j, unsigned long long best) { VT_ROW_KEYS(p.out, row, j)[cta] = best; });
+            if (lane == 0) VT_ROW_MS(p.out, row)[cta] = pack_ms(ms.x, ms.y);
+            __threadfence();
+            __syncwarp();
+            unsigned int ticket = 0;
+            if (lane == 0) ticket = atomicAdd(&p.out.hdr->row_ticket[row], 1u);
+            ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+            if (ticket == (unsigned int)G - 1u) {
+                __threadfence();
+                merge_row_global(p.out, G, row);
+                if (lane == 0) p.out.hdr->row_ticket[row] = 0u;        // ready for the next call
+            }
+        } else {
+            unsigned long long* dst = VT_REC(p.out, cta, p.m_begin + m);
+            warp_select_topk(rec0, stride, P1, k, cbuf, [&](int j, unsigned long long best) { dst[j] = best; });
+            if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
+        }
     }
 }
 
@@ -280,10 +290,6 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.stage_bytes = (uint32_t)sr * c.d * 2;
         const size_t h_bytes = ((size_t)MP * c.d * 2 + 127) & ~(size_t)127;
         const size_t list_bytes = ((size_t)kGemvConsumers * kGemvR * MP * KS * 8 + 127) & ~(size_t)127;
-        const size_t cand_bytes = (size_t)kGemvWarps * kMergeCand * 8;
-        size_t merge_bytes = (size_t)grid * (KS * 8 + 16) + cand_bytes;            // one row per batch at least
-        const size_t one_copy = (size_t)grid * ws_pitch(c.out.M, c.out.k) * 8 + cand_bytes;   // all rows in one copy
-        if (c.out.fused_merge && one_copy <= 128 * 1024) merge_bytes = std::max(merge_bytes, one_copy);
         const size_t bar_bytes = (size_t)(2 * 32 + 1) * 8 + 16;
         const size_t fold_bytes = (size_t)kGemvMaxM * kMergeCand * 8;
         const size_t fixed = h_bytes + list_bytes + fold_bytes + bar_bytes;
@@ -299,7 +305,6 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
         off += list_bytes;
         p.fold_off = (uint32_t)off;
         off += fold_bytes;
-        if (off < merge_bytes) off = (merge_bytes + 127) & ~(size_t)127;   // merge staging reuses [0, bar_off)
         p.bar_off = (uint32_t)off;
         p.total_smem = (uint32_t)(off + bar_bytes);
         if (p.total_smem > (uint32_t)kMaxDynSmem) return VT_ERR_UNSUPPORTED;
