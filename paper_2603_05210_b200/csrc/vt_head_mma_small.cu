@@ -21,12 +21,12 @@
 //              after the other would put several round trips to L2 per row on the critical path: the kernel then
 //              only writes the records and a one-warp-per-row merge kernel follows it.
 // Short tiles (a CTA with at most 64 rows: V_trim up to about 9,500) would waste the MMA: it costs the same 60-80
-// cycles for 28 live rows as for 128, and 4 * nk of them per tile is then what the call takes.  With M <= 8 the
-// kernel folds G = 4 (2) k-blocks into one MMA instead: TMEM lanes 32g..32g+31 (64g..) hold the tile's rows for
-// k-block G*j + g, and since an 8-row block of h per k-block is already laid out 1 KB after the other, a B
-// operand of N = 8 * G rows is the matching k-blocks of h.  Lane group g against column group g is the wanted
-// partial sum (the other G - 1 column groups are cross terms nobody reads); the readers add the G partial sums
-// through shared memory.  G times fewer MMAs per tile.
+// cycles for 28 live rows as for 128, and 4 * nk of them per tile is then what the call takes.  The kernel then
+// folds G = 4 (2) k-blocks into one MMA instead: TMEM lanes 32g..32g+31 (64g..) hold the tile's rows for
+// k-block G*j + g, and since the blocks of h for consecutive k-blocks lie one after the other (resident or in the
+// ring), a B operand of N = G * (rows of a block) rows is the matching k-blocks of h.  Lane group g against column
+// group g is the wanted partial sum (the other G - 1 column groups are cross terms nobody reads); the readers add
+// the G partial sums through shared memory.  G times fewer MMAs per tile.
 // The weight stream is the bound (arithmetic intensity = M FLOP/B).
 #include <cuda.h>
 
@@ -54,14 +54,15 @@ struct SmallParams {
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
     uint32_t tmem_cols;       // allocation: 2 accumulators of N columns, a power of two >= 32
     int d, nk;                // nk = 64-column k-blocks
-    int G;                    // k-blocks folded into one MMA: 128 / (tile height rounded up to 32 or 64), M <= 8 only, else 1
+    int G;                    // k-blocks folded into one MMA: 128 / (tile height rounded up to 32 or 64), or 1
+    int NG;                   // accumulator columns per folded k-block = rows of an h block: 8 (M <= 8), else M rounded up to 16
     int nsb;                  // MMA steps along d: ceil(nk / G) "super-blocks" of G k-blocks
     int TH;                   // vocabulary rows per tile (<= 128)
     int kb_per_stage;         // k-blocks one ring stage holds
     int n_stages;
     uint32_t slot_bytes;      // one k-block of a tile in the ring: TH rounded up to whole 8-row groups x 128 B
     uint32_t sub_bytes;       // with folded k-blocks: bytes between the k-blocks of one MMA step in a slot (128 / G rows x 128 B)
-    uint32_t part_off;        // with folded k-blocks: the readers' partial sums [G][8][64] floats
+    uint32_t part_off;        // with folded k-blocks: the readers' partial sums [G][NG][64] floats
     uint32_t blk_bytes;       // slot_bytes, plus h_blk when h rides in the ring (the h block follows the weights)
     uint32_t stage_bytes;
     uint32_t w_tx;            // bytes one W box delivers (TH * 128)
@@ -185,14 +186,16 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (*abort_flag) { ok = false; break; }
                     const int nb = min(kbs, nsb - ks);
                     const uint32_t bar = bar_full + 8u * s;
-                    mbar_arrive_expect_tx(bar, (uint32_t)nb * ((uint32_t)KF * p.w_tx + (p.h_resident ? 0u : p.h_blk)));
+                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + (p.h_resident ? 0u : p.h_blk)));
                     for (int kb = 0; kb < nb; ++kb) {
                         const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
                         // k-block KF * (ks + kb) + g goes to lanes g * (128 / KF) ...; one past d is all zero fill
                         for (int g = 0; g < KF; ++g)
                             tma_load_2d_hint(dst + (uint32_t)g * p.sub_bytes, &tmW, ((ks + kb) * KF + g) * kBoxK, row0, bar,
                                              stream_once);
-                        if (!p.h_resident) tma_load_2d(dst + p.slot_bytes, &tmH, (ks + kb) * kBoxK, 0, bar);
+                        if (!p.h_resident)          // the matching k-blocks of h, one block after the other behind the weights
+                            for (int g = 0; g < KF; ++g)
+                                tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK, 0, bar);
                     }
                     ++issued;
                     if (++s == S) { s = 0; ++wrap; }
@@ -280,27 +283,37 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 }
                 const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
                 if (KF > 1) {
-                    // Folded k-blocks: this warp's lanes are k-group g of tile rows r0 + lane, and columns 8g..8g+7
-                    // of the accumulator are their partial logits for the (up to 8) draft rows.
-                    const int SR = 128 / KF, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
+                    // Folded k-blocks: this warp's lanes are k-group g of tile rows r0 + lane, and columns
+                    // NG*g .. NG*g + NG - 1 of the accumulator are their partial logits for the draft rows.
+                    const int SR = 128 / KF, NG = p.NG, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
                     float* part = reinterpret_cast<float*>(smem + p.part_off);
                     if (got) {
                         tc_fence_after();
-                        uint32_t v[8];
-                        tc_ld8(taddr + (uint32_t)(8 * g), v);
-                        tc_wait_ld();
+                        if (NG == 8) {
+                            uint32_t v[8];
+                            tc_ld8(taddr + (uint32_t)(8 * g), v);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int m = 0; m < 8; ++m) part[(g * 8 + m) * 64 + r] = __uint_as_float(v[m]);
+                        } else {
+                            for (int c0 = 0; c0 < NG; c0 += 16) {
+                                uint32_t v[16];
+                                tc_ld16(taddr + (uint32_t)(NG * g + c0), v);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int m = 0; m < 16; ++m) part[(g * NG + c0 + m) * 64 + r] = __uint_as_float(v[m]);
+                            }
+                        }
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
-#pragma unroll
-                        for (int m = 0; m < 8; ++m) part[(g * 8 + m) * 64 + r] = __uint_as_float(v[m]);
                     }
                     reader_barrier();                                  // all four readers' partial sums are in place
                     for (int e = tid; e < M * SR; e += 128) {
                         const int m = e / SR, rr = e - m * SR;
                         if (rr >= nv) continue;
                         float sum = 0.0f;
-                        for (int gg = 0; gg < KF; ++gg) sum += part[(gg * 8 + m) * 64 + rr];
+                        for (int gg = 0; gg < KF; ++gg) sum += part[(gg * p.NG + m) * 64 + rr];
                         lg[m * kLgPitch + rr] = sum;
                         if (p.out.logits) p.out.logits[(size_t)m * Vt + row0 + rr] = sum;
                     }
@@ -395,21 +408,25 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     // h resident (M <= 8 only: 8 rows per k-block) when that still leaves a ring of four stages; else it streams
     for (int attempt = M <= 8 ? 0 : 1; attempt < 3; ++attempt) {
         const int resident = attempt == 0;
-        // short tiles with a resident 8-row h: fold G k-blocks into each MMA
-        p->G = !resident ? 1 : p->TH <= 32 ? 4 : p->TH <= 64 ? 2 : 1;
+        // short tiles: fold G k-blocks into each MMA, as far as the accumulator (G * NG columns) and the partial sums allow
+        p->NG = M <= 8 ? 8 : ((M + 15) / 16) * 16;            // = rows of one h block
+        p->G = p->TH <= 32 ? 4 : p->TH <= 64 ? 2 : 1;
+        // measured at d = 4096 with h in the ring: G = 4 gains (M = 16, 32 at 28 rows per CTA), G = 2 loses (M = 32 at 56
+        // rows, M = 48 and 64 at 28), so there it is four or nothing
+        if (!resident && (p->G < 4 || 4 * p->NG > 128)) p->G = 1;
         p->nsb = (p->nk + p->G - 1) / p->G;
-        p->N = p->G > 1 ? 8 * p->G : ((M + 15) / 16) * 16;
+        p->N = p->G > 1 ? p->NG * p->G : ((M + 15) / 16) * 16;
         p->sub_bytes = (uint32_t)(128 / p->G) * 128u;
         p->slot_bytes = p->G > 1 ? 16384u : (uint32_t)((p->TH + 7) / 8) * 1024u;
         p->tmem_cols = 32;
         while (p->tmem_cols < 2u * (uint32_t)p->N) p->tmem_cols *= 2;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 128
         p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const size_t part_bytes = p->G > 1 ? (size_t)p->G * 8 * 64 * 4 : 0;
+        const size_t part_bytes = p->G > 1 ? (size_t)p->G * p->NG * 64 * 4 : 0;
         // + zeros for what the last MMA step reads past h: rows 8-15 of an unfolded step, whole k-blocks of a folded one
         const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 * (size_t)p->G : 0;
         p->h_resident = resident;
-        p->blk_bytes = p->slot_bytes + (resident ? 0u : p->h_blk);
+        p->blk_bytes = p->slot_bytes + (resident ? 0u : (uint32_t)p->G * p->h_blk);
         // A stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height; two k-blocks at
         // least (four MMAs per hand-over are too few), one only as the last resort.
         p->kb_per_stage = std::max(2, std::min(4, (int)((28 * 1024 + p->blk_bytes / 2) / p->blk_bytes)));
