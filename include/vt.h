@@ -49,7 +49,8 @@ typedef enum vt_path {
     VT_PATH_AUTO = 0,      /* chosen from M and d                                                     */
     VT_PATH_GEMV = 1,      /* CUDA-core streaming GEMV; 4 draft rows per pass, d <= 8192              */
     VT_PATH_MMA = 2,       /* tcgen05 tensor-core GEMM, draft rows on the TMEM lanes; any M            */
-    VT_PATH_MMA_SMALL = 3  /* tcgen05 tensor-core GEMM, vocabulary rows on the TMEM lanes; M <= 64         */
+    VT_PATH_MMA_SMALL = 3  /* tcgen05 tensor-core GEMM, vocabulary rows on the TMEM lanes; any M, in passes
+                              of 128 draft rows                                                        */
 } vt_path;
 
 /* Text for a status code (static storage). */

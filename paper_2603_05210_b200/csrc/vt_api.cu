@@ -73,9 +73,8 @@ static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, 
 // Automatic path choice, from measurements at d = 4096 over V_trim = 4096 .. 128256:
 //  - the CUDA-core GEMV has the least fixed cost and keeps up with the stream for one draft row: M = 1 always,
 //    and M = 2 while the weights are under 80 MB, where fixed cost decides;
-//  - the vocabulary-rows-on-lanes tensor-core kernel for every other M <= 64;
-//  - the draft-rows-on-lanes tensor-core kernel for the rest.
-constexpr int kAutoSmallMaxM = 64;
+//  - the vocabulary-rows-on-lanes tensor-core kernel for everything else it can plan (passes of 128 draft rows);
+//  - the draft-rows-on-lanes tensor-core kernel for what it declines (very large k times M, very large d).
 static bool auto_prefers_gemv(int M, int d, int Vt) {
     if (!gemv_supports(d)) return false;
     const size_t w_bytes = (size_t)Vt * d * 2;
@@ -97,7 +96,7 @@ static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
         return VT_ERR_SHAPE;
     } else if (auto_prefers_gemv(c.M, c.d, c.Vt)) {
         r = launch_head_gemv(c, st, &grid);
-    } else if (c.M <= kAutoSmallMaxM && (r = launch_head_mma_small(c, st, &grid)) != VT_ERR_UNSUPPORTED) {
+    } else if ((r = launch_head_mma_small(c, st, &grid)) != VT_ERR_UNSUPPORTED) {
         merged = true;     // launched (or failed for a reason another path would not cure)
     } else {
         r = launch_head_mma(c, st, &grid);

@@ -38,7 +38,8 @@ namespace vt {
 
 constexpr int kSmMaxEpiWarps = 16;            // warps 0-7, or 0-15 when there are more than 8 draft rows; 0-3 also read TMEM
 constexpr int kSmThreads = (kSmMaxEpiWarps + 2) * 32;     // at most: the epilogue warps, then the producer, then the MMA issuer
-constexpr int kSmMaxM = 64;                   // draft rows <= MMA N <= 64
+constexpr int kSmMaxM = 128;                  // draft rows per launch <= MMA N <= 128
+constexpr int kLgRows = 32;                   // draft rows whose tile logits shared memory holds at a time
 constexpr int kSmMaxStages = 32;
 constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
 constexpr int kHParts = 4;                    // h arrives in this many parts so the first MMAs need not wait for all of it
@@ -46,7 +47,8 @@ constexpr int kSmCand = 128 + VT_MAX_K;       // candidate keys per epilogue war
 
 struct SmallParams {
     HeadOut out;
-    int M;                    // draft rows, <= kSmMaxM
+    int M;                    // draft rows of this launch, <= kSmMaxM
+    int m_begin;              // first of them among the call's draft rows
     int merge_in_kernel;      // 1: one draft row per epilogue warp, merged by the last warp to publish it; 0: a merge kernel follows
     int n_epi;                // epilogue warps: 8, or 16 when M > 8; the block has two more (producer, MMA issuer)
     uint32_t scratch_stride;  // bytes of one epilogue warp's candidate buffer: (128 + k) keys
@@ -195,7 +197,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                                              stream_once);
                         if (!p.h_resident)          // the matching k-blocks of h, one block after the other behind the weights
                             for (int g = 0; g < KF; ++g)
-                                tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK, 0, bar);
+                                tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK,
+                                            p.m_begin, bar);
                     }
                     ++issued;
                     if (++s == S) { s = 0; ++wrap; }
@@ -263,17 +266,18 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 if (k0 >= k1) break;
                 mbar_arrive_expect_tx(bar_h + 8u * j, (uint32_t)(k1 - k0) * p.h_blk);
                 for (int kb = k0; kb < k1; ++kb)
-                    tma_load_2d(base + p.h_off + (uint32_t)kb * p.h_blk, &tmH, kb * kBoxK, 0, bar_h + 8u * j);
+                    tma_load_2d(base + p.h_off + (uint32_t)kb * p.h_blk, &tmH, kb * kBoxK, p.m_begin, bar_h + 8u * j);
             }
         }
         __syncwarp();
         unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(scratch);
-        // Every epilogue warp passes the same two barriers per tile whatever happens, so none can be left
-        // waiting at one: after a wait has run out the remaining tiles only skip their work.
+        // Every epilogue warp passes the same barriers per tile whatever happens, so none can be left waiting at
+        // one: after a wait has run out the remaining tiles only skip their work.
         for (int t = 0; t < ntiles; ++t) {
             const int buf = t & 1;
             const int row0 = row_begin + t * TH;
             const int nv = min(TH, row_end - row0);
+            bool got_tile = false;
             if (warp < 4) {
                 // warp-uniform decisions: tcgen05.ld needs the whole warp
                 bool got = false;
@@ -315,61 +319,73 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         float sum = 0.0f;
                         for (int gg = 0; gg < KF; ++gg) sum += part[(gg * p.NG + m) * 64 + rr];
                         lg[m * kLgPitch + rr] = sum;
-                        if (p.out.logits) p.out.logits[(size_t)m * Vt + row0 + rr] = sum;
+                        if (p.out.logits) p.out.logits[(size_t)(p.m_begin + m) * Vt + row0 + rr] = sum;
                     }
-                } else if (got) {
-                    tc_fence_after();
+                }
+                got_tile = got;
+            }
+            // The tile's logits go through shared memory kLgRows draft rows at a time: readers lay a chunk out per
+            // draft row, every epilogue warp folds its rows of the chunk, and the buffer is free for the next chunk.
+            for (int c0 = 0; c0 < M; c0 += kLgRows) {
+                const int mc = min(kLgRows, M - c0);
+                if (warp < 4 && KF == 1 && got_tile) {
+                    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N + c0);
                     const int i = warp * 32 + lane;                    // TMEM lane = vocabulary row of the tile
-                    for (int c0 = 0; c0 < p.N; c0 += 16) {             // 16 draft rows at a time
+                    if (c0 == 0) tc_fence_after();
+                    for (int c1 = 0; c1 < mc; c1 += 16) {              // 16 draft rows per load
                         uint32_t r[16];
-                        tc_ld16(taddr + (uint32_t)c0, r);
+                        tc_ld16(taddr + (uint32_t)c1, r);
                         tc_wait_ld();
                         if (i < nv) {
 #pragma unroll
                             for (int m = 0; m < 16; ++m)
-                                if (c0 + m < M) lg[(c0 + m) * kLgPitch + i] = __uint_as_float(r[m]);
+                                if (c1 + m < mc) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(r[m]);
                             if (p.out.logits) {
 #pragma unroll
                                 for (int m = 0; m < 16; ++m)
-                                    if (c0 + m < M) p.out.logits[(size_t)(c0 + m) * Vt + row0 + i] = __uint_as_float(r[m]);
+                                    if (c1 + m < mc)
+                                        p.out.logits[(size_t)(p.m_begin + c0 + c1 + m) * Vt + row0 + i] = __uint_as_float(r[m]);
                             }
                         }
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                    if (c0 + kLgRows >= M) {                           // the accumulator is read out
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                    }
                 }
+                epi_barrier(n_epi * 32);                               // the chunk's logits are in shared memory
+                for (int m = c0 + warp; m < c0 + mc; m += n_epi) {
+                    const float tau = warp_topk_update<4>(lg + (m - c0) * kLgPitch, nv, row0, lists + (size_t)m * k, k,
+                                                          tau_s[m], cbuf, ms_s + m, lane);
+                    __syncwarp();
+                    if (lane == 0) tau_s[m] = tau;
+                    __syncwarp();
+                }
+                epi_barrier(n_epi * 32);                               // ... and may be overwritten
             }
-            epi_barrier(n_epi * 32);                                   // the tile's logits are in shared memory
-            for (int m = warp; m < M; m += n_epi) {
-                const float tau = warp_topk_update<4>(lg + m * kLgPitch, nv, row0, lists + (size_t)m * k, k, tau_s[m], cbuf,
-                                                      ms_s + m, lane);
-                __syncwarp();
-                if (lane == 0) tau_s[m] = tau;
-                __syncwarp();
-            }
-            epi_barrier(n_epi * 32);                                   // ... and may be overwritten
         }
         // ------------------------------------------------------------------ publish, and merge if last
         // The warp owns its rows from the first tile to the outputs: record -> fence -> ticket; the warp that
         // draws the last ticket of a row (over all CTAs) merges that row.  No CTA-wide step in between.
         for (int m = warp; m < M; m += n_epi) {
+            const int row = p.m_begin + m;                             // among the call's draft rows
             const unsigned long long* list = lists + (size_t)m * k;
-            for (int j = lane; j < k; j += 32) VT_ROW_KEYS(p.out, m, j)[cta] = list[j];
+            for (int j = lane; j < k; j += 32) VT_ROW_KEYS(p.out, row, j)[cta] = list[j];
             if (lane == 0) {
                 const float2 ms = ms_s[m];
-                VT_ROW_MS(p.out, m)[cta] = pack_ms(ms.x, ms.y);
+                VT_ROW_MS(p.out, row)[cta] = pack_ms(ms.x, ms.y);
             }
             if (!p.merge_in_kernel) continue;      // the records are complete when the kernel is
             __threadfence();
             __syncwarp();
             unsigned int ticket = 0;
-            if (lane == 0) ticket = atomicAdd(&p.out.hdr->row_ticket[m], 1u);
+            if (lane == 0) ticket = atomicAdd(&p.out.hdr->row_ticket[row], 1u);
             ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
             if (ticket == (unsigned int)G - 1u) {
                 __threadfence();
-                merge_row_global(p.out, G, m);
-                if (lane == 0) p.out.hdr->row_ticket[m] = 0u;          // ready for the next call
+                merge_row_global(p.out, G, row);
+                if (lane == 0) p.out.hdr->row_ticket[row] = 0u;        // ready for the next call
             }
         }
         if (warp == n_epi - 1 && lane == 0 && ntiles > 0 && p.h_resident && *abort_flag) {
@@ -397,7 +413,7 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     p->TH = (R + nt - 1) / nt;
     p->w_tx = (uint32_t)p->TH * 128u;
     p->h_blk = M <= 8 ? 1024u : (uint32_t)(((M + 15) / 16) * 16) * 128u;
-    const size_t lg_bytes = ((size_t)M * kLgPitch * 4 + 127) & ~(size_t)127;
+    const size_t lg_bytes = ((size_t)std::min(M, kLgRows) * kLgPitch * 4 + 127) & ~(size_t)127;
     const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
     p->n_epi = M > 8 ? kSmMaxEpiWarps : 8;
     p->merge_in_kernel = M <= p->n_epi;
@@ -461,10 +477,11 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     if (r != VT_OK) return r;
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
-    SmallParams p{};
-    if (!small_plan(c.M, c.d, c.Vt, c.out.k, grid, &p)) return VT_ERR_UNSUPPORTED;
-    p.out = c.out;
-
+    // every pass of kSmMaxM draft rows must fit before anything is launched
+    for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {
+        SmallParams q{};
+        if (!small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &q)) return VT_ERR_UNSUPPORTED;
+    }
     static int configured_device = -1;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
@@ -473,16 +490,25 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
         if (e != cudaSuccess) return cuda_fail(e);
         configured_device = dev;
     }
-    CUtensorMap tmW, tmH;
-    r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, p.TH);
-    if (r != VT_OK) return r;
-    r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
-    if (r != VT_OK) return r;
-    cudaError_t e = launch_pdl(head_mma_small_kernel, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
-    count_launch();
-    if (e == cudaSuccess) e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(e);
-    return p.merge_in_kernel ? VT_OK : launch_merge_rowmajor(c.out, grid, st);
+    bool merge_after = false;
+    for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {        // each pass streams the weights once for its draft rows
+        SmallParams p{};
+        small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p);
+        p.out = c.out;
+        p.m_begin = m0;
+        if (c.M > kSmMaxM) p.merge_in_kernel = 0;       // row tickets serve single-pass calls only
+        merge_after = !p.merge_in_kernel;
+        CUtensorMap tmW, tmH;
+        r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, p.TH);
+        if (r != VT_OK) return r;
+        r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
+        if (r != VT_OK) return r;
+        cudaError_t e = launch_pdl(head_mma_small_kernel, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
+        count_launch();
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return merge_after ? launch_merge_rowmajor(c.out, grid, st) : VT_OK;
 }
 
 }  // namespace vt

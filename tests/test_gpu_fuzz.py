@@ -41,7 +41,7 @@ def test_random_shape_both_paths(vt, oracle, M, d, Vt, k):
     h, W, d2t = rand_case(M, d, Vt, seed=M * 31 + d * 7 + Vt + k)
     ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
     Wd = dev_bf16(W)
-    paths = (vt.VT_PATH_AUTO, vt.VT_PATH_GEMV, vt.VT_PATH_MMA) + ((vt.VT_PATH_MMA_SMALL,) if M <= 64 else ())
+    paths = (vt.VT_PATH_AUTO, vt.VT_PATH_GEMV, vt.VT_PATH_MMA) + (vt.VT_PATH_MMA_SMALL,)
     for path in paths:
         got = run_head(vt, h, Wd, d2t, k, path)
         parity.check_head(got, ora, d2t, k)

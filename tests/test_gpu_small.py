@@ -32,12 +32,7 @@ def rand_case(M, d, Vt, seed, w_std=0.02, h_std=1.0):
 
 
 PATHS = [pytest.param(1, id="gemv"), pytest.param(2, id="mma"), pytest.param(3, id="mma_small")]
-SMALL_MAX_M = 64          # VT_PATH_MMA_SMALL takes at most this many draft rows
-
-
 def skip_unless_path_takes(path, M, d):
-    if path == 3 and M > SMALL_MAX_M:
-        pytest.skip("the few-draft-rows tensor-core path takes M <= 64")
     if path == 1 and d > 8192:
         pytest.skip("the GEMV path takes d <= 8192")
 
@@ -132,7 +127,8 @@ HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8)
                (8, 4096, 6521, 8), (2, 3072, 1000, 64), (9, 2048, 300, 10), (17, 128, 1025, 3),
                (4, 5120, 700, 8), (64, 512, 333, 10), (5, 200, 2000, 33), (1, 4096, 13264, 1),
                (16, 256, 40000, 10), (7, 64, 60001, 64), (12, 4096, 3000, 8), (2, 8192, 600, 5),
-               (33, 1024, 20000, 10), (64, 4096, 2500, 8), (48, 2048, 9000, 16), (8, 16384, 400, 4)]
+               (33, 1024, 20000, 10), (64, 4096, 2500, 8), (48, 2048, 9000, 16), (8, 16384, 400, 4),
+               (100, 2048, 30000, 10), (128, 512, 1000, 8), (257, 256, 20000, 3)]
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -212,19 +208,12 @@ def test_all_paths_agree_on_logits(vt):
 
 @pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (16, 1), (17, 2), (64, 2), (65, 2), (300, 4)])
 def test_launches_per_call_of_the_automatic_choice(vt, oracle, M, launches):
-    # M = 1: GEMV; M <= 16: one launch, rows merged by the last warp to publish them; M <= 64: the same kernel
-    # followed by the row-wise merge kernel; beyond: the draft-rows-on-lanes kernel in passes of 128 rows, then a merge
+    # M = 1: GEMV; M <= 16: one launch, rows merged by the last warp to publish them; beyond: the same kernel in
+    # passes of 128 draft rows followed by the row-wise merge kernel
     h, W, d2t = rand_case(M, 256, 3000, seed=40 + M)
     got = run_head(vt, h, dev_bf16(W), d2t, 4, vt.VT_PATH_AUTO)
     assert vt.vt_last_launch_count() == launches
     parity.check_head(got, oracle.draft_head(h, W, d2t, 4, want_logits=True), d2t, 4)
-
-
-def test_forced_small_path_refuses_many_draft_rows(vt):
-    h, W, d2t = rand_case(65, 64, 100, seed=12)
-    with pytest.raises(vt.VtError) as e:
-        run_head(vt, h, dev_bf16(W), d2t, 4, 3)
-    assert e.value.status == vt.VT_ERR_UNSUPPORTED
 
 
 def test_trimmed_head_equals_full_head_restricted(vt, oracle):
