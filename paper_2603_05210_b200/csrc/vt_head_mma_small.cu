@@ -1,10 +1,10 @@
-// Draft head, tensor-core path for few draft rows (M <= 64): vocabulary rows on the TMEM lanes.
+// Draft head, tensor-core path with the vocabulary rows on the TMEM lanes (any M, 128 draft rows per launch).
 //
 //   D[i, m] = sum_j W_trim[row0 + i, j] * h[m, j]       (the d -> k linear head, 2*d*k FLOPs per draft row)
 //
-// Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (N = 16, 32, 48 or
-// 64 rows: the draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes x N columns in
-// tensor memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
+// Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (N = M rounded up
+// to 16, at most 128 rows: the draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes
+// x N columns in tensor memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
 // row, so reading a tile out costs one instruction per thread whatever M is, and a weight tile needs no
 // padding rows: the tile height is the CTA's row count split evenly (<= 128), rows of the MMA past it compute
 // on stale shared memory and land in lanes nobody reads.  For M <= 8 h stays in shared memory for the whole
@@ -13,7 +13,8 @@
 //   next warp  TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
 //   last warp  MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
 //              ring stage; two accumulator buffers in TMEM
-//   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory
+//   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory,
+//              32 draft rows at a time
 //   warps 0-7  (0-15 when M > 8) warp w owns draft rows w, w + 8 (16), ...: running (max, sum-exp) and top-k of the row over the tile
 //              (warp_topk_update), and at the end the row's record, its arrival ticket and, for the warp that
 //              arrives last of all CTAs, the row's final merge (merge_row_global).  No CTA-wide barrier and no
