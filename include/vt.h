@@ -109,8 +109,17 @@ vt_status vt_validate_keep_ids(const int32_t* keep_ids, int V_trim, int V_full,
  *              an arrival counter and a status word; calls that share a workspace must be
  *              ordered on one stream.
  * d % 8 == 0, d >= 8; 1 <= k <= min(V_trim, VT_MAX_K); any M >= 1.  Inputs must be finite.
+ * W_trim is treated as a constant of the model: the kernels are launched with programmatic
+ *   dependent launch and may start streaming W_trim as soon as the stream's previous kernel lets
+ *   its dependents start, which for this library's own head kernels is while their last rows
+ *   are still being merged (h, d2t, the workspace and the outputs are only touched once the
+ *   previous kernel has completed).  A kernel without such an early trigger - vt_compact_head,
+ *   a cudaMemcpyAsync, any ordinary kernel - releases its dependents only when it has
+ *   finished, so producing W_trim with those earlier on the same stream is safe.  Do not
+ *   produce W_trim with a kernel that triggers its dependents before its last write to it.
  * Asynchronous: no host synchronisation.  A device-side wait that ran out is reported by
- * vt_last_status on the same workspace.
+ * vt_last_status on the same workspace; after VT_ERR_TIMEOUT run vt_workspace_init again before
+ * the workspace is reused (arrival counters may be left mid-count).
  */
 size_t    vt_workspace_bytes(int M, int k);
 vt_status vt_workspace_init(void* workspace, size_t workspace_bytes, void* stream);

@@ -164,9 +164,12 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above touched only shared memory, tensor memory and kernel parameters, so under programmatic
-    // dependent launch it overlaps the previous kernel's tail.  No thread reads or writes global memory before
-    // this wait (it returns once the previous kernel has completed and its writes are visible).
-    grid_dependency_wait();
+    // dependent launch it overlaps the previous kernel's tail.  Every thread but the producer now waits until the
+    // previous kernel has completed and its writes are visible; nothing of h, d2t, the workspace or the outputs is
+    // touched before that.  The producer does not wait: W_trim is a constant of the model (the header says what
+    // that asks of the caller), so its stream starts as soon as this CTA is resident - while the previous call
+    // still merges - and the ring is full when the first MMA may be issued.
+    if (warp != producer_warp) grid_dependency_wait();
     if (tid == 0) grid_launch_dependents();
 
     auto fail = [&]() {
