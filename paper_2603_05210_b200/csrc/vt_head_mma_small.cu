@@ -449,9 +449,14 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
         const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 * (size_t)p->G : 0;
         p->h_resident = resident;
         p->blk_bytes = p->slot_bytes + (resident ? 0u : (uint32_t)p->G * p->h_blk);
-        // A stage of 24-32 KB amortises the per-stage barrier hand-over whatever the tile height; two k-blocks at
-        // least (four MMAs per hand-over are too few), one only as the last resort.
+        // Every hand-over of a stage costs the issuing thread some 300 cycles beside its MMAs, and that thread is what
+        // limits how fast an SM can take weights: two k-blocks per stage at least (24-32 KB), and three where four
+        // such stages still fit and the tiles are tall (measured at 109-row tiles, d = 4096: 1-5 % faster than two;
+        // with only three stages left, or with folded short tiles, slower), one only as the last resort.
         p->kb_per_stage = std::max(2, std::min(4, (int)((28 * 1024 + p->blk_bytes / 2) / p->blk_bytes)));
+        if (p->G == 1 && p->kb_per_stage == 2 && p->nk >= 6 &&
+            common + h_bytes + part_bytes + 4 * (size_t)(3 * p->blk_bytes) <= (size_t)kMaxDynSmem)
+            p->kb_per_stage = 3;
         if (attempt == 2) p->kb_per_stage = 1;
         p->kb_per_stage = std::min(p->kb_per_stage, p->nsb);
         p->stage_bytes = p->blk_bytes * (uint32_t)p->kb_per_stage;
