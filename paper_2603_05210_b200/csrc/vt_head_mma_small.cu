@@ -4,23 +4,24 @@
 //
 // Operand roles: A = a tile of up to 128 vocabulary rows of W_trim (K-major as stored), B = h (N = M rounded up
 // to 16, at most 128 rows: the draft rows, zero-filled or don't-care beyond M), D = fp32 accumulator of 128 lanes
-// x N columns in tensor memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its logit for every draft
-// row, so reading a tile out costs one instruction per thread whatever M is, and a weight tile needs no
-// padding rows: the tile height is the CTA's row count split evenly (<= 128), rows of the MMA past it compute
-// on stale shared memory and land in lanes nobody reads.  Each k-block of h rides in the ring next to its weights
-// (it comes from L2: every CTA reads the same h); only with M <= 8 and short tiles does h stay in shared memory
-// for the whole kernel instead.
-//   next warp  TMA producer: boxes of 64 columns x tile-height rows of W into a shared-memory ring
-//   last warp  MMA issuer: four K=16 tcgen05.mma (M=128, N=16) per 64-column k-block, tcgen05.commit frees the
-//              ring stage; two accumulator buffers in TMEM
-//   warps 0-3  read TMEM (warp q: lanes 32q..32q+31) and lay the tile's logits out per draft row in shared memory,
-//              32 draft rows at a time
-//   warps 0-7  (0-15 when M > 8) warp w owns draft rows w, w + 8 (16), ...: running (max, sum-exp) and top-k of the row over the tile
-//              (warp_topk_update), and at the end the row's record, its arrival ticket and, for the warp that
-//              arrives last of all CTAs, the row's final merge (merge_row_global).  No CTA-wide barrier and no
-//              CTA ever waits for another.  With more than 16 draft rows a warp owns several, and merging them one
-//              after the other would put several round trips to L2 per row on the critical path: the kernel then
-//              only writes the records and a one-warp-per-row merge kernel follows it.
+// x N columns in tensor memory.  tcgen05.ld then hands each of 128 epilogue threads one vocabulary row and its
+// logits for 16 draft rows, so reading a tile out is cheap whatever M is, and a weight tile needs no padding rows:
+// the tile height is the CTA's row count split evenly (<= 128), rows of the MMA past it compute on stale shared
+// memory and land in lanes nobody reads.  Each k-block of h rides in the ring next to its weights (it comes from
+// L2: every CTA reads the same h); only with M <= 8 and short tiles does h stay in shared memory for the whole
+// kernel instead.
+//   warps 0-7   (0-15 when M > 8) the epilogue.  Warps 0-3 read TMEM (warp q: lanes 32q..32q+31) and lay the tile's
+//               logits out per draft row in shared memory, 32 draft rows at a time.  Warp w owns draft rows w,
+//               w + 8 (16), ...: running (max, sum-exp) and top-k of the row over the tile (warp_topk_update), at
+//               the end the row's record, and with at most 16 draft rows its arrival ticket and, for the warp that
+//               arrives last of all CTAs, the row's final merge (merge_row_global): no CTA-wide barrier and no CTA
+//               ever waits for another.  With more rows a warp owns several, and merging them one after the other
+//               would put several round trips to L2 per row on the critical path: the kernel then only writes
+//               the records and a one-warp-per-row merge kernel follows it.
+//   next warp   TMA producer: boxes of 64 columns x tile-height rows of W (and the k-block of h) into a
+//               shared-memory ring; it starts before the dependency wait (W_trim is a model constant)
+//   last warp   MMA issuer: four K=16 tcgen05.mma (M=128, N) per 64-column k-block, tcgen05.commit frees the ring
+//               stage; two accumulator buffers in TMEM
 // Short tiles (a CTA with at most 64 rows: V_trim up to about 9,500) would waste the MMA: it costs the same 60-80
 // cycles for 28 live rows as for 128, and 4 * nk of them per tile is then what the call takes.  The kernel then
 // folds G = 4 (2) k-blocks into one MMA instead: TMEM lanes 32g..32g+31 (64g..) hold the tile's rows for
