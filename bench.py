@@ -313,6 +313,9 @@ def run_ours(args):
     if rank == 0 and world == 1:
         if not args.no_curve:
             line["curve"] = latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, not args.no_graph)
+            del W_full
+            torch.cuda.empty_cache()
+            line["other_workloads"] = config_timings(vt, torch, l2, peak_gbs, not args.no_graph)
         line["cpu_baseline"] = cpu_baseline(case)
     if rank == 0:
         print(json.dumps(line))
@@ -341,6 +344,36 @@ def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, use_graph=True
             out.append({"V_trim": Vt, "M": M, "us_per_call": round(us, 2), "GBs": round(gbs, 1),
                         "frac": round(gbs / peak_gbs, 4)})
         del copies, W_trim
+        torch.cuda.empty_cache()
+    return out
+
+
+def config_timings(vt, torch, l2, peak_gbs, use_graph=True):
+    """us/call of the other benchmark workloads (shapes of the five configurations; random device-side weights,
+    since only the shapes matter for the time).  The 95 % prefix of the fifth follows the input recipe."""
+    V = inputs.V_LLAMA3
+    tokens = inputs.zipf_token_stream(V, 1.05, 10_000_000, 5000)
+    _, sorted_counts = inputs.frequency_ranking(tokens, V)
+    vt95 = int(inputs.smallest_prefix_with_coverage(sorted_counts, 19, 20))
+    shapes = [("cfg1", 2048, 4096, 1, 1)]
+    shapes += [("cfg2", 3072, v, 1, 1) for v in (4096, 8192, 16384, 32000, V)]
+    shapes += [("cfg4", 4096, 16384, m, 10) for m in (16, 64, 256)]
+    shapes += [("cfg5 trimmed to 95 % coverage", 5120, vt95, 32, 8), ("cfg5 untrimmed", 5120, V, 32, 8)]
+    out = []
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    for name, d, Vt, M, k in shapes:
+        free, _ = torch.cuda.mem_get_info()
+        nc = n_copies_for_cold(Vt * d * 2, l2, free)
+        copies = [(torch.randn((Vt, d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16) for _ in range(nc)]
+        h = torch.randn((M, d), device="cuda", generator=gen).to(torch.bfloat16)
+        d2t = torch.arange(Vt, dtype=torch.int32, device="cuda")
+        steps = 480 if Vt * d <= 32000 * 4096 else 120
+        ms, launches = time_head(vt, torch, h, copies, d2t, k, steps, 20, use_graph=use_graph)
+        us = ms * 1000.0 / steps
+        gbs = head_bytes(d, Vt, M, k) / (us * 1e-6) / 1e9
+        out.append({"config": name, "d": d, "V_trim": Vt, "M": M, "k": k, "us_per_call": round(us, 2),
+                    "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4), "launches_per_call": launches})
+        del copies
         torch.cuda.empty_cache()
     return out
 
