@@ -53,6 +53,15 @@ typedef enum vt_path {
                               of 128 draft rows                                                        */
 } vt_path;
 
+#define VT_PATH_MASK 0xFF  /* the vt_path part of an `options` argument */
+
+/* Option bits for vt_draft_head_path, ORed onto the vt_path value. */
+#define VT_HEAD_STATIC_WEIGHTS 0x100 /* the caller declares W_trim a constant of the model: nothing earlier in the
+                                        stream writes it (see vt_draft_head).  The kernels may then request weights
+                                        ahead of the stream-order dependency wait.                                 */
+#define VT_HEAD_D2T_OFFSETS    0x200 /* d2t holds offsets instead of ids: target id = draft index + d2t[draft index],
+                                        the form an EAGLE-3 style checkpoint stores (Section 1)                     */
+
 /* Text for a status code (static storage). */
 const char* vt_strerror(vt_status s);
 
@@ -109,14 +118,16 @@ vt_status vt_validate_keep_ids(const int32_t* keep_ids, int V_trim, int V_full,
  *              an arrival counter and a status word; calls that share a workspace must be
  *              ordered on one stream.
  * d % 8 == 0, d >= 8; 1 <= k <= min(V_trim, VT_MAX_K); any M >= 1.  Inputs must be finite.
- * W_trim is treated as a constant of the model: the kernels are launched with programmatic
- *   dependent launch and may start streaming W_trim as soon as the stream's previous kernel lets
- *   its dependents start, which for this library's own head kernels is while their last rows
- *   are still being merged (h, d2t, the workspace and the outputs are only touched once the
- *   previous kernel has completed).  A kernel without such an early trigger - vt_compact_head,
- *   a cudaMemcpyAsync, any ordinary kernel - releases its dependents only when it has
- *   finished, so producing W_trim with those earlier on the same stream is safe.  Do not
- *   produce W_trim with a kernel that triggers its dependents before its last write to it.
+ * Stream order: the kernels are launched with programmatic dependent launch, i.e. their CTAs may become
+ *   resident while the stream's previous kernel is finishing (for this library's own head kernels: while
+ *   their last rows are still being merged).  They set up shared and tensor memory and then wait for that
+ *   kernel to complete before they touch h, W_trim, d2t, the workspace or the outputs, so every input may be
+ *   produced by earlier work on the same stream, whatever kind of kernel produced it.
+ *   vt_draft_head_path with VT_HEAD_STATIC_WEIGHTS relaxes this for W_trim only: the caller declares that
+ *   nothing earlier in the stream writes W_trim (it was written once, e.g. by vt_compact_head, and the
+ *   stream or device was synchronised afterwards - the usual state of model weights in a serving loop).
+ *   Weight tiles are then requested before the wait, which hides the first memory round trip behind the
+ *   previous call's tail.  h, d2t, the workspace and the outputs keep full stream-order semantics.
  * Asynchronous: no host synchronisation.  A device-side wait that ran out is reported by
  * vt_last_status on the same workspace; after VT_ERR_TIMEOUT run vt_workspace_init again before
  * the workspace is reused (arrival counters may be left mid-count).
@@ -130,13 +141,15 @@ vt_status vt_draft_head(const void* h, const void* W_trim, const int32_t* d2t,
                         int32_t* draft_ids, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream);
 
-/* Same call with the contraction kernel forced (VT_ERR_UNSUPPORTED if that kernel cannot take
- * the shape).  VT_PATH_AUTO is what vt_draft_head uses. */
+/* Same call with options: `options` = a vt_path value (a forced contraction kernel returns
+ * VT_ERR_UNSUPPORTED if it cannot take the shape; VT_PATH_AUTO is what vt_draft_head uses), optionally ORed
+ * with VT_HEAD_STATIC_WEIGHTS and / or VT_HEAD_D2T_OFFSETS.  vt_draft_head is this call with options = 0.
+ * Unknown option bits give VT_ERR_SHAPE. */
 vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d2t,
                              int M, int d, int V_trim, int k,
                              int32_t* target_ids, float* logprobs,
                              int32_t* draft_ids, float* lse,
-                             void* workspace, size_t workspace_bytes, void* stream, int path);
+                             void* workspace, size_t workspace_bytes, void* stream, int options);
 
 /* End-to-end form of vt_draft_head for callers whose per-step data lives on the host:
  * h_host (host [M, d] bf16, ideally pinned) is copied to the device, the head runs, and
@@ -192,7 +205,8 @@ vt_status vt_coverage(const int32_t* token_ids, int64_t N,
  *   cum_counts dev [V_full] uint64 (out) or NULL: cum_counts[k-1] = occurrences covered by the top k
  *   k_star     host (out);  C_star, R_star, U_star  host (out), each may be NULL
  *   workspace  dev, 256-byte aligned, vt_select_workspace_bytes(V_full); contents are overwritten
- * 1 <= k_min <= k_max <= V_full, 0 <= alpha <= 1, F_fixed >= 0, d >= 1.  SYNCHRONISES the stream.
+ * 1 <= k_min <= k_max <= V_full, 0 <= alpha <= 1, F_fixed >= 0, d >= 1, N < 2^32 (frequencies are counted in
+ * 32 bits; a longer stream gives VT_ERR_SHAPE).  SYNCHRONISES the stream.
  * VT_ERR_EMPTY if N == 0 or no id falls inside [0, V_full). */
 size_t    vt_select_workspace_bytes(int V_full);
 vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed,
@@ -215,8 +229,9 @@ vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d
  *  - V_full may be at most 262,144 (the built-in bitmap is 32 KiB; with its counters the array takes
  *    33,024 bytes on every device that loads the library, until the process ends).  A larger V_full
  *    returns VT_ERR_SHAPE and launches nothing.
- *  - The first call on a device looks up the array's device address and remembers it.  Make that first
- *    call on each device outside any stream capture.
+ *  - The first call on a device looks up the array's device address and remembers it.
+ *  - Every call ends by synchronising the stream to read the count back, so it cannot be part of a stream
+ *    capture at all (neither can vt_coverage).
  *  - All calls on a device share the one array.  Each call clears it before use, so results do not
  *    depend on earlier calls, but two calls whose GPU work can overlap (different streams, different
  *    host threads) race on it: keep them ordered.
@@ -241,17 +256,30 @@ vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V
 vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
                    int32_t* target_ids, void* stream);
 
-/* The index buffers an EAGLE-3 style draft stores with its weights (Section 1: "draft-to-target and
- * target-to-draft index buffers"), derived from keep_ids:
+/* The two index buffers an EAGLE-3 style draft stores with its weights (the draft-to-target and the
+ * target-to-draft map of Section 1), derived from keep_ids:
  *   d2t_offsets[i] = keep_ids[i] - i        (target id = draft index + offset), dev [V_trim] int32 or NULL
  *   t2d_mask[v]    = 1 if v is kept else 0,                                      dev [V_full] uint8 or NULL
- * At least one output must be given.  The head calls above take absolute ids (keep_ids itself as d2t); this
- * call only converts for checkpoints that use the offset form.  Asynchronous. */
+ * At least one output must be given.  The head calls above take absolute ids (keep_ids itself as d2t) unless
+ * VT_HEAD_D2T_OFFSETS is set, in which case they take the d2t_offsets this call writes.  Asynchronous. */
 vt_status vt_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full,
                         int32_t* d2t_offsets, uint8_t* t2d_mask, void* stream);
 
 /* Number of kernels the last call of this thread launched (for launch accounting). */
 int vt_last_launch_count(void);
+
+/* Failure-path probe: one tiny kernel posts an mbarrier transaction that no copy will ever complete and
+ * waits on it with the same bounded wait the head kernels use, limited to `limit_us` microseconds
+ * (1 .. 1,000,000).  When the limit runs out it sets the time-out bit in the workspace's status word and
+ * exits normally - nothing is in flight, nothing faults - so vt_last_status(workspace) then reports
+ * VT_ERR_TIMEOUT, exactly as after a head call whose wait ran out.  workspace: a draft-head workspace.
+ * Asynchronous. */
+vt_status vt_test_timeout_probe(void* workspace, int limit_us, void* stream);
+
+/* Stream-order probe: a kernel that releases its programmatic dependents at once, idles for `delay_us`
+ * microseconds (0 .. 10,000) and only then copies n_bytes (a multiple of 16; dev pointers, 16-byte aligned)
+ * from src to dst.  A head call enqueued right behind it must still see the copied bytes. Asynchronous. */
+vt_status vt_test_late_copy(void* dst, const void* src, size_t n_bytes, int delay_us, void* stream);
 
 #ifdef __cplusplus
 }

@@ -14,7 +14,8 @@ _BINDING_NAMES = {
     "vt_coverage", "vt_coverage_static", "vt_select_vocab", "vt_select_workspace_bytes", "vt_debug_logits", "vt_remap", "vt_vocab_maps", "vt_last_launch_count",
     "VT_OK", "VT_ERR_NULL", "VT_ERR_SHAPE", "VT_ERR_ALIGN", "VT_ERR_RANGE", "VT_ERR_DUP", "VT_ERR_EMPTY",
     "VT_ERR_WORKSPACE", "VT_ERR_TIMEOUT", "VT_ERR_CUDA", "VT_ERR_UNSUPPORTED", "VT_MAX_K",
-    "VT_PATH_AUTO", "VT_PATH_GEMV", "VT_PATH_MMA", "VT_PATH_MMA_SMALL",
+    "VT_PATH_AUTO", "VT_PATH_GEMV", "VT_PATH_MMA", "VT_PATH_MMA_SMALL", "VT_HEAD_STATIC_WEIGHTS", "VT_HEAD_D2T_OFFSETS",
+    "vt_test_timeout_probe", "vt_test_late_copy",
 }
 
 

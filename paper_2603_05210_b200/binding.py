@@ -20,6 +20,7 @@ VT_ERR_NULL, VT_ERR_SHAPE, VT_ERR_ALIGN, VT_ERR_RANGE, VT_ERR_DUP = 1, 2, 3, 4, 
 VT_ERR_EMPTY, VT_ERR_WORKSPACE, VT_ERR_TIMEOUT, VT_ERR_CUDA, VT_ERR_UNSUPPORTED = 6, 7, 8, 9, 10
 VT_MAX_K = 64
 VT_PATH_AUTO, VT_PATH_GEMV, VT_PATH_MMA, VT_PATH_MMA_SMALL = 0, 1, 2, 3
+VT_HEAD_STATIC_WEIGHTS, VT_HEAD_D2T_OFFSETS = 0x100, 0x200
 
 # every symbol include/vt.h declares: name -> (restype, argtypes)
 _p, _i, _i64, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
@@ -45,6 +46,8 @@ SYMBOLS = {
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
     "vt_vocab_maps": (_i, [_p, _i, _i, _p, _p, _p]),
     "vt_last_launch_count": (_i, []),
+    "vt_test_timeout_probe": (_i, [_p, _i, _p]),
+    "vt_test_late_copy": (_i, [_p, _p, _sz, _i, _p]),
 }
 
 _lib = None
@@ -150,8 +153,11 @@ def vt_validate_keep_ids(keep_ids: torch.Tensor, V_full: int, workspace: torch.T
 def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, d2t: torch.Tensor, k: int, *,
                   workspace: torch.Tensor | None = None, path: int = VT_PATH_AUTO,
                   target_ids: torch.Tensor | None = None, logprobs: torch.Tensor | None = None,
-                  draft_ids: torch.Tensor | None = None, lse: torch.Tensor | None = None):
-    """(target_ids [M,k] int32, logprobs [M,k] float32); pass ``draft_ids`` / ``lse`` tensors to receive those too."""
+                  draft_ids: torch.Tensor | None = None, lse: torch.Tensor | None = None,
+                  static_weights: bool = False, d2t_offsets: bool = False):
+    """(target_ids [M,k] int32, logprobs [M,k] float32); pass ``draft_ids`` / ``lse`` tensors to receive those too.
+
+    ``static_weights`` sets VT_HEAD_STATIC_WEIGHTS, ``d2t_offsets`` sets VT_HEAD_D2T_OFFSETS (see ``include/vt.h``)."""
     h = _bf16(h, "h")
     W_trim = _bf16(W_trim, "W_trim")
     d2t = _i32(d2t, "d2t")
@@ -167,7 +173,9 @@ def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, d2t: torch.Tensor, k: i
         logprobs = torch.empty((M, k), dtype=torch.float32, device=h.device)
     _check(lib().vt_draft_head_path(h.data_ptr(), W_trim.data_ptr(), d2t.data_ptr(), M, d, Vt, k,
                                     target_ids.data_ptr(), logprobs.data_ptr(), _ptr(draft_ids), _ptr(lse),
-                                    workspace.data_ptr(), workspace.numel(), _stream(), path), "vt_draft_head")
+                                    workspace.data_ptr(), workspace.numel(), _stream(),
+                                    path | (VT_HEAD_STATIC_WEIGHTS if static_weights else 0)
+                                    | (VT_HEAD_D2T_OFFSETS if d2t_offsets else 0)), "vt_draft_head")
     return target_ids, logprobs
 
 
@@ -275,3 +283,14 @@ def vt_vocab_maps(keep_ids: torch.Tensor, V_full: int) -> tuple[torch.Tensor, to
 
 def vt_last_launch_count() -> int:
     return int(lib().vt_last_launch_count())
+
+
+def vt_test_timeout_probe(workspace: torch.Tensor, limit_us: int) -> None:
+    _check(lib().vt_test_timeout_probe(workspace.data_ptr(), int(limit_us), _stream()), "vt_test_timeout_probe")
+
+
+def vt_test_late_copy(dst: torch.Tensor, src: torch.Tensor, delay_us: int) -> None:
+    n = src.numel() * src.element_size()
+    if dst.numel() * dst.element_size() != n:
+        raise ValueError("dst and src differ in size")
+    _check(lib().vt_test_late_copy(dst.data_ptr(), src.data_ptr(), n, int(delay_us), _stream()), "vt_test_late_copy")

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libvt.so")
-SOURCES = ["vt_api.cu", "vt_aux.cu", "vt_head_gemv.cu", "vt_head_mma.cu", "vt_head_mma_small.cu", "vt_merge.cu", "vt_select.cu"]
+SOURCES = ["vt_api.cu", "vt_aux.cu", "vt_head_gemv.cu", "vt_head_mma.cu", "vt_head_mma_small.cu", "vt_merge.cu", "vt_probe.cu", "vt_select.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -1,4 +1,5 @@
 // C entry points: argument checks on the host, path choice, launches.  See include/vt.h for the contract.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -18,20 +19,36 @@ vt_status driver_fail(int cu_result) {
     return VT_ERR_CUDA;
 }
 void count_launch() { ++g_launches; }
+void reset_launch_count() { g_launches = 0; }
 
 vt_status device_sm_count(int* sms) {
-    static int cached[64];
+    static std::atomic<int> cached[64];       // zero-initialised; racing first calls store the same value
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
-    if (cached[dev] == 0) {
-        int n = 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
         e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return cuda_fail(e);
-        cached[dev] = n;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    *sms = cached[dev];
+    *sms = n;
+    return VT_OK;
+}
+
+// Raises a kernel's dynamic shared-memory limit once per device (an atomic bit per device: concurrent host
+// threads may both make the call, which is harmless).
+vt_status ensure_max_dyn_smem(const void* kernel, int bytes, std::atomic<unsigned long long>* done_mask) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
+    const unsigned long long bit = 1ull << dev;
+    if (done_mask->load(std::memory_order_acquire) & bit) return VT_OK;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+    done_mask->fetch_or(bit, std::memory_order_release);
     return VT_OK;
 }
 
@@ -52,9 +69,10 @@ static vt_status check_head_args(const void* h, const void* W, const int32_t* d2
 constexpr int kFusedMergeMaxM = 16;
 
 static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, float* lp, int32_t* did, float* lse,
-                        float* logits, void* ws) {
+                        float* logits, void* ws, int d2t_offsets = 0) {
     HeadOut o{};
     o.d2t = d2t;
+    o.d2t_offsets = d2t_offsets;
     o.target_ids = tid;
     o.logprobs = lp;
     o.draft_ids = did;
@@ -188,13 +206,16 @@ vt_status vt_workspace_init(void* workspace, size_t workspace_bytes, void* strea
 
 vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d2t, int M, int d, int V_trim, int k,
                              int32_t* target_ids, float* logprobs, int32_t* draft_ids, float* lse, void* workspace,
-                             size_t workspace_bytes, void* stream, int path) {
+                             size_t workspace_bytes, void* stream, int options) {
     g_launches = 0;
     vt_status r = check_head_args(h, W_trim, d2t, M, d, V_trim, k, target_ids, logprobs, workspace, workspace_bytes);
     if (r != VT_OK) return r;
+    if (options & ~(VT_PATH_MASK | VT_HEAD_STATIC_WEIGHTS | VT_HEAD_D2T_OFFSETS)) return VT_ERR_SHAPE;
     HeadCall c{h, W_trim, d, M, V_trim,
-               make_out(d2t, M, V_trim, k, target_ids, logprobs, draft_ids, lse, nullptr, workspace)};
-    return run_head(c, (cudaStream_t)stream, path);
+               make_out(d2t, M, V_trim, k, target_ids, logprobs, draft_ids, lse, nullptr, workspace,
+                        (options & VT_HEAD_D2T_OFFSETS) ? 1 : 0),
+               (options & VT_HEAD_STATIC_WEIGHTS) ? 1 : 0};
+    return run_head(c, (cudaStream_t)stream, options & VT_PATH_MASK);
 }
 
 vt_status vt_draft_head(const void* h, const void* W_trim, const int32_t* d2t, int M, int d, int V_trim, int k,
@@ -243,7 +264,7 @@ vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32
     }
     cudaError_t e = cudaMemcpyAsync(h_dev, h_host, (size_t)M * d * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
-    HeadCall c{h_dev, W_trim, d, M, V_trim, make_out(d2t, M, V_trim, k, tid_out, lp_out, nullptr, nullptr, nullptr, workspace)};
+    HeadCall c{h_dev, W_trim, d, M, V_trim, make_out(d2t, M, V_trim, k, tid_out, lp_out, nullptr, nullptr, nullptr, workspace), 0};
     r = run_head(c, st, VT_PATH_AUTO);
     if (r != VT_OK) return r;
     if (!direct) {
@@ -311,8 +332,8 @@ vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V
     vt_status r = check_head_args(h, W_trim, tid, M, d, V_trim, 1, tid, lp, workspace, head_ws);
     if (r != VT_OK) return r;
     HeadOut o = make_out(nullptr, M, V_trim, 1, tid, lp, nullptr, nullptr, logits, workspace);
-    HeadCall c{h, W_trim, d, M, V_trim, o};
-    return run_head(c, (cudaStream_t)stream, path);
+    HeadCall c{h, W_trim, d, M, V_trim, o, 0};
+    return run_head(c, (cudaStream_t)stream, path & VT_PATH_MASK);
 }
 
 vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim, int32_t* target_ids,

@@ -195,15 +195,9 @@ vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full,
     const size_t words = coverage_bitmap_words(V_full);
     const int in_smem = words * 4 <= kCoverageSmemBitmapMax;
     const size_t smem = in_smem ? words * 4 : 0;
-    static int configured_device = -1;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
-    if (configured_device != dev) {
-        cudaError_t e = cudaFuncSetAttribute(coverage_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kCoverageSmemBitmapMax);
-        if (e != cudaSuccess) return cuda_fail(e);
-        configured_device = dev;
-    }
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(coverage_count_kernel), (int)((int)kCoverageSmemBitmapMax), &smem_configured); rc != VT_OK)
+        return rc;
     const long long per_cta = (long long)kCoverageThreads * 4 * 8;   // ids one CTA takes in 8 trips
     const int grid = (int)std::max(1LL, std::min((N + per_cta - 1) / per_cta, (long long)sms * 2));
     coverage_count_kernel<<<grid, kCoverageThreads, smem, st>>>(token_ids, N, V_full, bitmap, (int)words, in_smem,
@@ -224,18 +218,18 @@ static __device__ __align__(256) unsigned char g_static_coverage[sizeof(Coverage
 // handle for the runtime, not a pointer a kernel could use, so the address is asked for once per device
 // (with that device current) and remembered.
 static vt_status static_coverage_address(void** out) {
-    static void* cached[64];
+    static std::atomic<void*> cached[64];     // racing first calls on a device look up and store the same address
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev < 0 || dev >= 64) return cuda_fail(cudaErrorInvalidDevice);
-    if (!cached[dev]) {
-        void* ptr = nullptr;
+    void* ptr = cached[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress(&ptr, g_static_coverage);
         if (e != cudaSuccess) return cuda_fail(e);
-        cached[dev] = ptr;
+        cached[dev].store(ptr, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = ptr;
     return VT_OK;
 }
 
@@ -244,6 +238,7 @@ static vt_status static_coverage_address(void** out) {
 extern "C" vt_status vt_coverage_static(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim,
                                         int V_full, uint64_t* covered_out, double* fraction_out, void* stream) {
     using namespace vt;
+    reset_launch_count();
     if (!keep_ids || (!token_ids && N > 0)) return VT_ERR_NULL;
     if (V_full < 1 || V_trim < 1 || N < 0) return VT_ERR_SHAPE;
     if (V_full > kStaticCoverageMaxV) return VT_ERR_SHAPE;       // the built-in scratch holds no larger bitmap

@@ -59,6 +59,7 @@ __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
 
 struct HeadOut {
     const int32_t* d2t;   // null: report draft indices as target ids
+    int d2t_offsets;      // 1: d2t holds offsets, target id = draft index + d2t[draft index]
     int32_t* target_ids;
     float* logprobs;
     int32_t* draft_ids;   // may be null
@@ -108,15 +109,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Waits for the phase with the given parity to complete, for at most kWaitLimitNs.
-// Returns false when the limit ran out (the caller records it and unwinds; nothing spins forever).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Waits for the phase with the given parity to complete, for at most `limit_ns` (one second unless the caller
+// asks for less).  Returns false when the limit ran out (the caller records it and unwinds; nothing spins forever).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
     for (int i = 0; i < 64; ++i)                       // the common case: no clock read on the way
         if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if (((++spins) & 0xFFu) == 0 && global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (((++spins) & 0xFFu) == 0 && global_timer_ns() - t0 > limit_ns) return false;
+    }
+    return true;
+}
+// The same wait against an absolute deadline (a %globaltimer value): an unwinding CTA that lets several copies
+// land shares one deadline between them instead of granting each its own second.
+__device__ __forceinline__ bool mbar_wait_until(uint32_t bar, uint32_t parity, unsigned long long deadline_ns) {
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if (((++spins) & 0x3Fu) == 0 && global_timer_ns() > deadline_ns) return false;
     }
     return true;
 }
@@ -416,7 +426,7 @@ __device__ __forceinline__ void write_winner(const HeadOut& o, int m, int j, uns
     const size_t out = (size_t)m * o.k + j;
     if (best != 0ull) {
         const int idx = key_index(best);
-        o.target_ids[out] = o.d2t ? __ldg(&o.d2t[idx]) : idx;
+        o.target_ids[out] = o.d2t ? (o.d2t_offsets ? idx + __ldg(&o.d2t[idx]) : __ldg(&o.d2t[idx])) : idx;
         o.logprobs[out] = key_logit(best) - lse;
         if (o.draft_ids) o.draft_ids[out] = idx;
     } else {   // fewer than k candidates exist only if a wait ran out upstream
@@ -572,8 +582,10 @@ __device__ inline void merge_rows(const HeadOut& o, int P, int m_begin, int m_co
             for (int p = threadIdx.x; p < P; p += blockDim.x)
                 bulk_g2s(smem_u32(stage + (size_t)p * stride), VT_REC(o, p, m_begin + b0), bytes, bar);
         }
-        if (!mbar_wait(bar, phase)) {
-            atomicOr(&o.hdr->status, kStatusTimeout);
+        // every thread takes the same decision, so none is left alone at the barrier that ends the batch
+        const bool timed_out = !mbar_wait(bar, phase);
+        if (__syncthreads_or(timed_out ? 1 : 0)) {
+            if (timed_out) atomicOr(&o.hdr->status, kStatusTimeout);
             break;
         }
         for (int r = warp; r < nb; r += nwarps)

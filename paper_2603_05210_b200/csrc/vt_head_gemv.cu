@@ -32,6 +32,7 @@ struct GemvParams {
     const uint16_t* W;       // [Vt, d] bf16
     HeadOut out;
     int m_begin, m_count;    // draft rows of this pass
+    int early_weights;       // 1: the first stages may be requested before the dependency wait (W_trim declared constant)
     int d;
     int rows_per_stage;      // multiple of kGemvR
     int n_stages;            // multiple of n_cons, so a stage is always consumed by the same warp
@@ -115,10 +116,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         bulk_g2s(smem_u32(smem) + (uint32_t)s * p.stage_bytes, p.W + (size_t)(row_begin + t * SR) * d, bytes,
                  bar_full + 8u * s);
     };
-    // Nothing above touched global memory.  W_trim is a constant of the model (the header says what that asks of
-    // the caller), so the producer starts the first stages before the wait below, while the previous kernel
-    // finishes; h, the workspace and the outputs are only touched after it.
-    const int prefilled = min(min(S, ntiles), kGemvPrefill);
+    // Nothing above touched global memory.  When the caller has declared W_trim a constant of the model, the
+    // producer starts the first stages before the wait below, while the previous kernel finishes; h, the
+    // workspace and the outputs are only touched after it.
+    const int prefilled = p.early_weights ? min(min(S, ntiles), kGemvPrefill) : 0;
     if (tid == 0)
         for (int t = 0; t < prefilled; ++t) issue_tile(t);
     grid_dependency_wait();
@@ -145,8 +146,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
                 issued = t + 1;
             }
             if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
+                const unsigned long long deadline = global_timer_ns() + kWaitLimitNs;
                 for (int t = max(0, issued - S); t < issued; ++t)
-                    (void)mbar_wait(bar_full + 8u * (t % S), (uint32_t)(t / S) & 1u);
+                    (void)mbar_wait_until(bar_full + 8u * (t % S), (uint32_t)(t / S) & 1u, deadline);
             }
         }
     } else {
@@ -261,14 +263,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
 template <int MP>
 static vt_status launch_one(const GemvParams& p, int grid, cudaStream_t st) {
     auto kern = head_gemv_kernel<MP>;
-    static int configured_device = -1;   // per instantiation
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
-    if (configured_device != dev) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-        if (e != cudaSuccess) return cuda_fail(e);
-        configured_device = dev;
-    }
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(kern), (int)(kMaxDynSmem), &smem_configured); rc != VT_OK)
+        return rc;
     cudaError_t e = launch_pdl(kern, grid, kGemvThreads, p.total_smem, st, p);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
@@ -296,6 +293,7 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
         p.out = c.out;
         p.m_begin = m0;
         p.m_count = mc;
+        p.early_weights = c.static_weights;
         p.d = c.d;
         int sr = 16384 / (2 * c.d);
         sr = std::max(kGemvR, std::min(16, sr) / kGemvR * kGemvR);

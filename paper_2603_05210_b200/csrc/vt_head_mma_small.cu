@@ -58,6 +58,7 @@ struct SmallParams {
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
     uint32_t tmem_cols;       // allocation: 2 accumulators of N columns, a power of two >= 32
     int d, nk;                // nk = 64-column k-blocks
+    int early_weights;        // 1: weight boxes may be requested before the dependency wait (W_trim declared constant)
     int G;                    // k-blocks folded into one MMA: 128 / (tile height rounded up to 32 or 64), or 1
     int NG;                   // accumulator columns per folded k-block = rows of an h block: 8 (M <= 8), else M rounded up to 16
     int nsb;                  // MMA steps along d: ceil(nk / G) "super-blocks" of G k-blocks
@@ -167,10 +168,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     // Everything above touched only shared memory, tensor memory and kernel parameters, so under programmatic
     // dependent launch it overlaps the previous kernel's tail.  Every thread but the producer now waits until the
     // previous kernel has completed and its writes are visible; nothing of h, d2t, the workspace or the outputs is
-    // touched before that.  The producer does not wait: W_trim is a constant of the model (the header says what
-    // that asks of the caller), so its stream starts as soon as this CTA is resident - while the previous call
-    // still merges - and the ring is full when the first MMA may be issued.
-    if (warp != producer_warp) grid_dependency_wait();
+    // touched before that.  The producing thread waits inside its own branch: when the caller has declared W_trim
+    // a constant of the model it first fills the ring with weight boxes - while the previous call still merges -
+    // so that the ring is full when the first MMA may be issued.
+    if (!(warp == producer_warp && lane == 0)) grid_dependency_wait();
     if (tid == 0) grid_launch_dependents();
 
     auto fail = [&]() {
@@ -181,37 +182,51 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     if (warp == producer_warp) {
         // ------------------------------------------------------------------ TMA producer: the weight stream
         if (lane == 0) {
-            int s = 0, issued = 0;
-            uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
-            bool ok = true;
             const int kbs = p.kb_per_stage;
+            const int spt = (nsb + kbs - 1) / kbs;          // ring stages per tile
+            const int total = ntiles * spt;                 // ring stages of this CTA, in issue order
             const uint64_t stream_once = l2_policy_evict_first();
-            for (int t = 0; t < ntiles && ok; ++t) {
+            const uint32_t h_tx = p.h_resident ? 0u : p.h_blk;
+            // stage q of the CTA's sequence into ring slot s: the weight boxes and/or the matching blocks of h
+            auto issue = [&](int q, int s, bool weights, bool hidden) {
+                const int t = q / spt, ks = (q - t * spt) * kbs;
                 const int row0 = row_begin + t * TH;
-                for (int ks = 0; ks < nsb; ks += kbs) {
-                    if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); ok = false; break; }
-                    if (*abort_flag) { ok = false; break; }
-                    const int nb = min(kbs, nsb - ks);
-                    const uint32_t bar = bar_full + 8u * s;
-                    mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + (p.h_resident ? 0u : p.h_blk)));
-                    for (int kb = 0; kb < nb; ++kb) {
-                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
-                        // k-block KF * (ks + kb) + g goes to lanes g * (128 / KF) ...; one past d is all zero fill
+                const int nb = min(kbs, nsb - ks);
+                const uint32_t bar = bar_full + 8u * s;
+                if (weights) mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + h_tx));
+                for (int kb = 0; kb < nb; ++kb) {
+                    const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
+                    // k-block KF * (ks + kb) + g goes to lanes g * (128 / KF) ...; one past d is all zero fill
+                    if (weights)
                         for (int g = 0; g < KF; ++g)
                             tma_load_2d_hint(dst + (uint32_t)g * p.sub_bytes, &tmW, ((ks + kb) * KF + g) * kBoxK, row0, bar,
                                              stream_once);
-                        if (!p.h_resident)          // the matching k-blocks of h, one block after the other behind the weights
-                            for (int g = 0; g < KF; ++g)
-                                tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK,
-                                            p.m_begin, bar);
-                    }
-                    ++issued;
-                    if (++s == S) { s = 0; ++wrap; }
+                    if (hidden && !p.h_resident)      // the matching k-blocks of h, one block after the other behind the weights
+                        for (int g = 0; g < KF; ++g)
+                            tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK,
+                                        p.m_begin, bar);
                 }
+            };
+            // With weights the caller declared constant, the ring is filled with weight boxes ahead of the
+            // dependency wait - each stage's barrier already expects the bytes of its h blocks, which are only
+            // requested after the wait, like every other read of what the previous kernel may have written.
+            const int pre = p.early_weights ? min(S, total) : 0;
+            for (int q = 0; q < pre; ++q) issue(q, q, true, false);
+            grid_dependency_wait();
+            for (int q = 0; q < pre; ++q) issue(q, q, false, true);
+            int s = pre == S ? 0 : pre, issued = pre;
+            uint32_t wrap = pre == S ? 1u : 0u;  // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
+            for (int q = pre; q < total; ++q) {
+                if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); break; }
+                if (*abort_flag) break;
+                issue(q, s, true, true);
+                ++issued;
+                if (++s == S) { s = 0; ++wrap; }
             }
             if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
+                const unsigned long long deadline = global_timer_ns() + kWaitLimitNs;
                 for (int i = max(0, issued - S); i < issued; ++i)
-                    (void)mbar_wait(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u);
+                    (void)mbar_wait_until(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u, deadline);
             }
         }
     } else if (warp == mma_warp) {
@@ -395,7 +410,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         }
         if (warp == n_epi - 1 && lane == 0 && ntiles > 0 && p.h_resident && *abort_flag) {
             // let the copies of h land before the CTA gives its shared memory back
-            for (int j = 0; j < kHParts && j * h_part < nk; ++j) (void)mbar_wait(bar_h + 8u * j, 0u);
+            const unsigned long long deadline = global_timer_ns() + kWaitLimitNs;
+            for (int j = 0; j < kHParts && j * h_part < nk; ++j) (void)mbar_wait_until(bar_h + 8u * j, 0u, deadline);
         }
     }
 
@@ -494,20 +510,16 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
         SmallParams q{};
         if (!small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &q)) return VT_ERR_UNSUPPORTED;
     }
-    static int configured_device = -1;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
-    if (configured_device != dev) {
-        cudaError_t e = cudaFuncSetAttribute(head_mma_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-        if (e != cudaSuccess) return cuda_fail(e);
-        configured_device = dev;
-    }
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel), (int)(kMaxDynSmem), &smem_configured); rc != VT_OK)
+        return rc;
     bool merge_after = false;
     for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {        // each pass streams the weights once for its draft rows
         SmallParams p{};
         small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p);
         p.out = c.out;
         p.m_begin = m0;
+        p.early_weights = c.static_weights;
         if (c.M > kSmMaxM) p.merge_in_kernel = 0;       // row tickets serve single-pass calls only
         merge_after = !p.merge_in_kernel;
         CUtensorMap tmW, tmH;

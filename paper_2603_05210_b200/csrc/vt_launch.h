@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <utility>
 
 #include "vt_common.cuh"
@@ -18,11 +19,14 @@ struct HeadCall {
     const void* W;
     int d, M, Vt;
     HeadOut out;
+    int static_weights;   // 1: the caller declared W_trim constant; its stream may start ahead of the dependency wait
 };
 
 vt_status cuda_fail(cudaError_t e);        // records e for vt_last_cuda_error, returns VT_ERR_CUDA
 vt_status driver_fail(int cu_result);
 void count_launch();
+void reset_launch_count();                  // every entry point starts with it, so vt_last_launch_count is per call
+vt_status ensure_max_dyn_smem(const void* kernel, int bytes, std::atomic<unsigned long long>* done_mask);
 vt_status device_sm_count(int* sms);
 
 // Both head kernels split the vocabulary rows over `*grid` persistent CTAs (one per SM at most); the
@@ -51,7 +55,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, siz
 bool gemv_supports(int d);
 vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid);
 vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid);
-// M <= 64; merges in the same launch for M <= 16, else launches the row-wise merge kernel after itself;
+// any M, in passes of 128 draft rows; a single pass of at most 16 rows merges row by row in the same launch (one
+// arrival ticket per draft row), everything else launches the row-wise merge kernel after itself;
 // VT_ERR_UNSUPPORTED when the shape does not fit
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid);
 vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st);

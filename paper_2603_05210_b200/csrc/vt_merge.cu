@@ -31,14 +31,9 @@ vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st) {
     if (want > cap) want = std::max(one_row, cap / one_row * one_row);
     want += cand;
     if (want > (size_t)kMaxDynSmem - 1024) return VT_ERR_UNSUPPORTED;
-    static int configured_device = -1;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
-    if (configured_device != dev) {
-        cudaError_t e = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem - 1024);
-        if (e != cudaSuccess) return cuda_fail(e);
-        configured_device = dev;
-    }
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(merge_kernel), (int)(kMaxDynSmem - 1024), &smem_configured); rc != VT_OK)
+        return rc;
     const int grid = (o.M + kMergeRowsPerCta - 1) / kMergeRowsPerCta;
     cudaError_t e = launch_pdl(merge_kernel, grid, kMergeThreads, want, st, o, P, (uint32_t)want);
     count_launch();

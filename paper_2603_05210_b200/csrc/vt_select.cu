@@ -219,7 +219,9 @@ extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_
                                      double c_min, int k_min, int k_max, int32_t* ranked_ids, uint64_t* cum_counts,
                                      int* k_star, double* C_star, double* R_star, double* U_star, void* workspace,
                                      size_t workspace_bytes, void* stream) {
+    reset_launch_count();
     if (!ranked_ids || !k_star || (!token_ids && N > 0)) return VT_ERR_NULL;
+    if (N > 0xFFFFFFFFll) return VT_ERR_SHAPE;                 // the histogram counts in 32 bits
     if (V_full < 1 || d < 1 || N < 0 || k_min < 1 || k_max < k_min || k_max > V_full || !(alpha >= 0.0 && alpha <= 1.0) ||
         !(F_fixed >= 0.0))
         return VT_ERR_SHAPE;
