@@ -33,7 +33,9 @@ METRIC = "draft_head_us_per_call"
 UNIT = "us/call"
 WORKLOAD = dict(d=4096, V_full=inputs.V_LLAMA3, V_trim=32000, M=8, k=8, seed=3000)
 WORKLOAD_NAME = "d=4096, V_trim=32000 of V_full=128256, M=8, top-k=8, log-softmax over V_trim, d2t remap"
-CURVE_VT = (4096, 8192, 16384, 32000, 128256)
+CURVE_VT = (4096, 4380, 6521, 8192, 13264, 16384, 32000, 128256)   # incl. the paper's vocabulary sizes (Sections 2.6, 3.2)
+REPS = 5              # repetitions of the timed region (median, spread and a 95 % interval are reported)
+ISOLATED_CALLS = 200  # single calls timed one by one behind an unrelated kernel
 CURVE_M = (1, 2, 4, 8, 16, 32, 64)
 FALLBACK_HBM_GBS = 6650.0
 
@@ -140,9 +142,19 @@ def to_dev(a, torch, dtype=None):
 GRAPH_CALLS = 120     # calls per captured CUDA graph (a multiple of every copy count the bench uses: 2..6, 8, 10, 12...)
 
 
-def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=True):
-    """CUDA-event time of exactly `steps` back-to-back calls rotating over W_copies; returns (ms total, launches/call).
+def stats(xs):
+    """median, 10th / 90th percentile and the 95 % interval of the mean of a list of samples."""
+    a = np.asarray(xs, dtype=np.float64)
+    half = 1.96 * float(a.std(ddof=1)) / np.sqrt(a.size) if a.size > 1 else 0.0
+    return {"median": round(float(np.median(a)), 3), "p10": round(float(np.percentile(a, 10)), 3),
+            "p90": round(float(np.percentile(a, 90)), 3), "mean": round(float(a.mean()), 3),
+            "ci95": [round(float(a.mean()) - half, 3), round(float(a.mean()) + half, 3)], "n": int(a.size)}
 
+
+def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=True, reps=1, static_weights=False):
+    """CUDA-event times of `reps` regions of exactly `steps` back-to-back calls rotating over W_copies.
+
+    Returns (ms of the first region if reps == 1 else the list of ms per region, launches per call).
     With use_graph the calls are replayed from a captured CUDA graph of GRAPH_CALLS calls (plus directly
     launched calls for the remainder), the way a serving loop would issue them; otherwise every call goes
     through the Python binding.  Either way each call is a separate kernel launch on the stream.
@@ -154,7 +166,8 @@ def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=T
     n = len(W_copies)
 
     def call(i):
-        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp,
+                         static_weights=static_weights)
 
     for i in range(warmup):
         call(i)
@@ -171,17 +184,47 @@ def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=T
                     call(i)
         torch.cuda.current_stream().wait_stream(side)
         graph.replay()                                   # one untimed replay: graph upload
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(n_replay):
-        graph.replay()
-    for i in range(steps - n_replay * GRAPH_CALLS):
-        call(i)
-    e1.record()
-    torch.cuda.synchronize()
+    out = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n_replay):
+            graph.replay()
+        for i in range(steps - n_replay * GRAPH_CALLS):
+            call(i)
+        e1.record()
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1))
     assert vt.vt_last_status(ws) == vt.VT_OK, "a device-side wait ran out during the timed region"
-    return e0.elapsed_time(e1), launches
+    return (out[0] if reps == 1 else out), launches
+
+
+def time_isolated(vt, torch, h, W_copies, d2t, k, n_calls=ISOLATED_CALLS, path=0):
+    """us of ONE call that follows an unrelated, ordinary kernel (an elementwise update of a 32 MB tensor: no
+    programmatic early trigger, and it displaces part of L2), timed with a CUDA event pair per call on a cold
+    copy of W_trim; the list of n_calls samples.  This is what a draft step sees inside a serving loop, where
+    the head follows the decoder layer and not another head call."""
+    M = h.shape[0]
+    ws = vt.new_workspace(vt.vt_workspace_bytes(M, k))
+    tid = torch.empty((M, k), dtype=torch.int32, device="cuda")
+    lp = torch.empty((M, k), dtype=torch.float32, device="cuda")
+    filler = torch.zeros(8 << 20, dtype=torch.float32, device="cuda")
+    n = len(W_copies)
+    for i in range(5):
+        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+    pairs = []
+    torch.cuda.synchronize()
+    for i in range(n_calls):
+        filler.add_(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    assert vt.vt_last_status(ws) == vt.VT_OK
+    return [a.elapsed_time(b) * 1000.0 for a, b in pairs]
 
 
 def n_copies_for_cold(bytes_per_copy, l2_bytes, free_bytes):
@@ -222,50 +265,40 @@ def run_ours(args):
     h = to_dev(case.h.view(np.int16), torch, torch.bfloat16)
     tok_dev = to_dev(tokens, torch)
 
-    # once-per-model steps: compaction (a1) and coverage (a6)
+    # once-per-model steps: compaction (a1), coverage (a6), vocabulary selection
     W_trim = vt.vt_compact_head(W_full, keep)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(10):
-        vt.vt_compact_head(W_full, keep, out=W_trim)
-    e1.record()
-    torch.cuda.synchronize()
-    compact_us = e0.elapsed_time(e1) * 100.0
-    cov_ws = torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda")
-    vt.vt_coverage(tok_dev, keep, V, cov_ws)
-    t0 = time.perf_counter()
-    for _ in range(10):
-        covered, frac = vt.vt_coverage(tok_dev, keep, V, cov_ws)
-    coverage_us = (time.perf_counter() - t0) * 1e5
-    # the paper's selection step (Eq. 1-5 as an exhaustive scan) on the same stream, Table 1 constants
-    F_fixed = 2.0 * (3 * d) * d + 436.2e6 + 50.3e6
-    sel_ws = torch.empty(vt.vt_select_workspace_bytes(V), dtype=torch.uint8, device="cuda")
-    sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
-    t0 = time.perf_counter()
-    for _ in range(5):
-        sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
-    select_us = (time.perf_counter() - t0) * 2e5
+    once = once_per_model(vt, torch, W_full, keep, W_trim, tok_dev, tokens, d, V, peak_gbs) if rank == 0 else {}
 
     free, _ = torch.cuda.mem_get_info()
     nc = n_copies_for_cold(W_trim.numel() * 2, l2, free)
     copies = [W_trim] + [W_trim.clone() for _ in range(nc - 1)]
 
-    # ---- timed region: K calls, device-timed, max over ranks
+    # ---- timed region: REPS x K calls, device-timed, max over ranks; the headline is the median region
     sampler = ClockSampler(local)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    ms, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup, use_graph=not args.no_graph)
+    ms_list, launches_per_call = time_head(vt, torch, h, copies, d2t, k, args.steps, args.warmup,
+                                           use_graph=not args.no_graph, reps=REPS)
     clocks = sampler.stop()
-    ms = max_over_ranks(ms, dist, "cuda")
+    ms_list = [max_over_ranks(x, dist, "cuda") for x in ms_list]
     if dist is not None:
         dist.barrier()
-    us_per_call_rank = ms * 1000.0 / args.steps
+    us_list = [x * 1000.0 / args.steps for x in ms_list]
+    us_per_call_rank = float(np.median(us_list))
+    ms = us_per_call_rank * args.steps / 1000.0
     value = whole_job_us_per_call(us_per_call_rank, world)
     bytes_call = head_bytes(d, Vt, M, k)
     achieved = bytes_call / (us_per_call_rank * 1e-6) / 1e9
+
+    # the same region with W_trim declared constant (VT_HEAD_STATIC_WEIGHTS): weights requested ahead of the
+    # stream-order wait; and single calls behind an unrelated kernel (what a serving loop sees)
+    ms_static, _ = time_head(vt, torch, h, copies, d2t, k, args.steps, min(args.warmup, 50), use_graph=not args.no_graph,
+                             reps=REPS, static_weights=True)
+    us_static = float(np.median([max_over_ranks(x, dist, "cuda") for x in ms_static])) * 1000.0 / args.steps
+    iso = time_isolated(vt, torch, h, copies, d2t, k)
+    us_iso = max_over_ranks(float(np.median(iso)), dist, "cuda")
 
     # ---- end to end: host h -> device, head, outputs -> host, every step
     e2e_steps = max(1, min(args.steps, 2000))
@@ -286,28 +319,32 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 6), "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAME if args.m is None else WORKLOAD_NAME.replace("M=8", f"M={M}"), "cold": f"calls rotate over {nc} copies of W_trim "
-                   f"({nc * W_trim.numel() * 2 / 1e6:.0f} MB >= 4x L2 of {l2 / 1e6:.0f} MB): inputs larger than L2",
-                   "step": "one vt_draft_head call (contraction + top-k + log-softmax + remap, one launch)",
-                   "launch": "eager calls through the binding" if args.no_graph or args.steps < GRAPH_CALLS
-                   else f"CUDA-graph replay of {GRAPH_CALLS}-call graphs (one kernel launch per call)",
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "calls_per_s": round(1e6 / value, 1)},
+        "config": bench_config(WORKLOAD_NAME if args.m is None else WORKLOAD_NAME.replace("M=8", f"M={M}"),
+                               cold=f"calls rotate over {nc} copies of W_trim ({nc * W_trim.numel() * 2 / 1e6:.0f} MB >= 4x L2 of "
+                                    f"{l2 / 1e6:.0f} MB): inputs larger than L2",
+                               step="one vt_draft_head call (contraction + top-k + log-softmax + remap, one launch), default options",
+                               launch="eager calls through the binding" if args.no_graph or args.steps < GRAPH_CALLS
+                               else f"CUDA-graph replay of {GRAPH_CALLS}-call graphs (one kernel launch per call)",
+                               parallelism="replicas only" if world > 1 else "single GPU",
+                               calls_per_s=round(1e6 / value, 1)),
+        "repetitions": {"regions": REPS, "us_per_call": stats(us_list), "value_is": "median region"},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak_gbs, "unit": "GB/s",
                      "frac": round(achieved / peak_gbs, 4), "of": peak_kind, "traffic": None if args.m is not None else ncu_traffic_or_none(),
                      "algorithmic_bytes_per_launch": bytes_call, "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
-                     "kernel": "head kernel of the chosen path; duration = timed region / launches"},
+                     "frac_isolated": round(bytes_call / (us_iso * 1e-6) / 1e9 / peak_gbs, 4),
+                     "frac_static_weights": round(bytes_call / (us_static * 1e-6) / 1e9 / peak_gbs, 4),
+                     "kernel": "head kernel of the chosen path; duration = timed region / launches (back-to-back calls); "
+                               "frac_isolated = the same bytes over the single-call latency below"},
+        "isolated_call": {"us": stats(iso), "calls": len(iso),
+                          "how": "CUDA events around one call that follows an unrelated elementwise kernel, cold W_trim copy"},
+        "static_weights": {"us_per_call": round(us_static / world, 3),
+                           "how": "same region with VT_HEAD_STATIC_WEIGHTS (W_trim declared constant: weight tiles are "
+                                  "requested ahead of the stream-order wait)"},
         "clocks": clocks,
         "e2e": {"value": round(e2e_us / world, 3), "unit": UNIT, "h2d_bytes_per_step": M * d * 2,
                 "d2h_bytes_per_step": M * k * 8, "steps": e2e_steps},
         "gpu_launches": args.steps * launches_per_call,
-        "once_per_model": {"compact_us": round(compact_us, 2),
-                           "compact_GBs": round(2 * W_trim.numel() * 2 / compact_us / 1e3, 1),
-                           "coverage_us_incl_sync": round(coverage_us, 2), "coverage_tokens": int(tokens.size),
-                           "coverage": frac,
-                           "select_vocab_us_incl_sync": round(select_us, 1),
-                           "select_vocab": {"alpha": 0.5, "c_min": 0.9, "k_range": [1000, 64000], "k_star": sel["k_star"],
-                                            "C": round(sel["C"], 6), "R": round(sel["R"], 6), "U": round(sel["U"], 6)}},
+        "once_per_model": once,
     }
 
     if rank == 0 and world == 1:
@@ -323,8 +360,77 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def bench_config(workload, cold, step, launch, parallelism, calls_per_s):
+    """Both arms print the same keys, so that their configurations can be compared field by field."""
+    return {"workload": workload, "cold": cold, "step": step, "launch": launch, "parallelism": parallelism,
+            "calls_per_s": calls_per_s}
+
+
+def event_us(torch, fn, reps):
+    """Median CUDA-event time of fn() in us, one event pair per call, after one untimed call."""
+    fn()
+    pairs = []
+    torch.cuda.synchronize()
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    return float(np.median([a.elapsed_time(b) for a, b in pairs])) * 1000.0
+
+
+def once_per_model(vt, torch, W_full, keep, W_trim, tok_dev, tokens, d, V, peak_gbs):
+    """The steps that run once per model: head compaction (row gather: read + write of the kept rows) at the bench
+    size and at the untrimmed size, the coverage count (Eq. 2: one read of the token stream) on the 1M- and a
+    10M-token stream, and the paper's selection step.  Device-timed; each with its own roofline fraction."""
+    out = {}
+    Vt = keep.numel()
+    us = event_us(torch, lambda: vt.vt_compact_head(W_full, keep, out=W_trim), 10)
+    gbs = 4 * d * Vt / us / 1e3
+    out["compact"] = [{"V_trim": Vt, "d": d, "us": round(us, 2), "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4),
+                       "bytes": 4 * d * Vt, "bound": "hbm read + write"}]
+    ident = torch.arange(V, dtype=torch.int32, device="cuda")
+    big = torch.empty_like(W_full)
+    us = event_us(torch, lambda: vt.vt_compact_head(W_full, ident, out=big), 5)
+    gbs = 4 * d * V / us / 1e3
+    out["compact"].append({"V_trim": V, "d": d, "us": round(us, 2), "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4),
+                           "bytes": 4 * d * V, "bound": "hbm read + write"})
+    del big
+    torch.cuda.empty_cache()
+    cov_ws = torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda")
+    covered, frac = vt.vt_coverage(tok_dev, keep, V, cov_ws)
+    out["coverage_value"] = frac
+    out["coverage"] = []
+    tok10 = torch.from_numpy(inputs.zipf_token_stream(V, 1.05, 10_000_000, 5000)).cuda()
+    for t in (tok_dev, tok10):
+        n = t.numel()
+        us = event_us(torch, lambda: vt.vt_coverage_enqueue(t, keep, V, cov_ws), 20)
+        gbs = 4 * n / us / 1e3
+        out["coverage"].append({"tokens": n, "us": round(us, 2), "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4),
+                                "bytes": 4 * n, "what": "bitmap clear + bitmap build + count (3 stream operations), no host read"})
+    t0 = time.perf_counter()
+    for _ in range(10):
+        vt.vt_coverage(tok_dev, keep, V, cov_ws)
+    out["coverage_us_incl_sync"] = round((time.perf_counter() - t0) * 1e5, 2)
+    del tok10
+    # the paper's selection step (Eq. 1-5 as an exhaustive scan) on the same stream, Table 1 constants
+    F_fixed = 2.0 * (3 * d) * d + 436.2e6 + 50.3e6
+    sel_ws = torch.empty(vt.vt_select_workspace_bytes(V), dtype=torch.uint8, device="cuda")
+    sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
+    t0 = time.perf_counter()
+    for _ in range(5):
+        sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
+    out["select_vocab_us_incl_sync"] = round((time.perf_counter() - t0) * 2e5, 1)
+    out["select_vocab"] = {"alpha": 0.5, "c_min": 0.9, "k_range": [1000, 64000], "k_star": sel["k_star"],
+                           "C": round(sel["C"], 6), "R": round(sel["R"], 6), "U": round(sel["U"], 6)}
+    return out
+
+
 def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, use_graph=True):
-    """us/call and roofline fraction over V_trim x M at d=4096 (the measured latency-vs-vocabulary curve)."""
+    """us/call and roofline fraction over V_trim x M at d=4096 (the measured latency-vs-vocabulary curve): back-to-back
+    calls (graph replay) and, beside them, single calls behind an unrelated kernel."""
     d, k = case.d, 8
     order = ranking[0]
     out = []
@@ -340,9 +446,12 @@ def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, use_graph=True
             steps = 480 if Vt <= 32000 else 120
             ms, _ = time_head(vt, torch, h, copies, keep, kk, steps, 20, use_graph=use_graph)
             us = ms * 1000.0 / steps
-            gbs = head_bytes(d, Vt, M, kk) / (us * 1e-6) / 1e9
+            us_iso = float(np.median(time_isolated(vt, torch, h, copies, keep, kk, n_calls=60)))
+            by = head_bytes(d, Vt, M, kk)
+            gbs = by / (us * 1e-6) / 1e9
             out.append({"V_trim": Vt, "M": M, "us_per_call": round(us, 2), "GBs": round(gbs, 1),
-                        "frac": round(gbs / peak_gbs, 4)})
+                        "frac": round(gbs / peak_gbs, 4), "us_isolated": round(us_iso, 2),
+                        "frac_isolated": round(by / (us_iso * 1e-6) / 1e9 / peak_gbs, 4)})
         del copies, W_trim
         torch.cuda.empty_cache()
     return out
@@ -370,16 +479,39 @@ def config_timings(vt, torch, l2, peak_gbs, use_graph=True):
         steps = 480 if Vt * d <= 32000 * 4096 else 120
         ms, launches = time_head(vt, torch, h, copies, d2t, k, steps, 20, use_graph=use_graph)
         us = ms * 1000.0 / steps
-        gbs = head_bytes(d, Vt, M, k) / (us * 1e-6) / 1e9
-        out.append({"config": name, "d": d, "V_trim": Vt, "M": M, "k": k, "us_per_call": round(us, 2),
-                    "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4), "launches_per_call": launches})
+        us_iso = float(np.median(time_isolated(vt, torch, h, copies, d2t, k, n_calls=60)))
+        by = head_bytes(d, Vt, M, k)
+        gbs = by / (us * 1e-6) / 1e9
+        row = {"config": name, "d": d, "V_trim": Vt, "M": M, "k": k, "us_per_call": round(us, 2),
+               "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4), "us_isolated": round(us_iso, 2),
+               "frac_isolated": round(by / (us_iso * 1e-6) / 1e9 / peak_gbs, 4), "launches_per_call": launches}
+        if M >= 128:      # where the tensor pipe is co-limiting: the contraction's share of the dense bf16 peak
+            row["TFLOPs"] = round(2.0 * M * d * Vt / (us * 1e-6) / 1e12, 1)
+        out.append(row)
         del copies
         torch.cuda.empty_cache()
     return out
 
 
+ONE_THREAD_SNIPPET = """
+import sys, time, numpy as np
+sys.path.insert(0, {root!r})
+import oracle
+from paper_2603_05210_b200 import inputs
+rows, d, M, k, seed = {rows}, {d}, {M}, {k}, {seed}
+W = inputs.normal_bf16((rows, d), 0.02, seed)
+h = inputs.hidden_states_bf16(M, d, seed, row_scale=(0.5, 2.0))
+d2t = np.arange(rows, dtype=np.int32)
+best = 1e30
+for _ in range(2):
+    t0 = time.perf_counter(); oracle.draft_head(h, W, d2t, k); best = min(best, time.perf_counter() - t0)
+print(oracle.num_threads(), best)
+"""
+
+
 def cpu_baseline(case):
-    """The oracle as it stands, timed on this host on the bench workload (best of 3 full calls)."""
+    """The oracle as it stands, timed on this host on the bench workload: one full call on all cores (best of 3),
+    and on one thread on a sample of the vocabulary rows scaled to the full call."""
     import oracle
     W_trim = oracle.compact(case.W_full, case.keep_ids)
     best = float("inf")
@@ -387,8 +519,21 @@ def cpu_baseline(case):
         t0 = time.perf_counter()
         oracle.draft_head(case.h, W_trim, case.d2t, case.k)
         best = min(best, time.perf_counter() - t0)
-    return {"value": round(best * 1e6, 1), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "the whole bench workload, one full call, best of 3"}
+    out = {"value": round(best * 1e6, 1), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": "the whole bench workload, one full call, best of 3"}
+    rows = 2000
+    try:
+        env = dict(os.environ, OMP_NUM_THREADS="1")
+        r = subprocess.run([sys.executable, "-c", ONE_THREAD_SNIPPET.format(root=ROOT, rows=rows, d=case.d, M=case.M, k=case.k,
+                                                                           seed=WORKLOAD["seed"])],
+                           capture_output=True, text=True, env=env, timeout=300)
+        nthreads, t = r.stdout.split()[-2:]
+        out["one_thread"] = {"value": round(float(t) * 1e6 * case.V_trim / rows, 1), "unit": UNIT, "cores": int(nthreads),
+                             "sample": f"the first {rows} of {case.V_trim} vocabulary rows (all {case.M} draft rows), "
+                                       f"scaled by {case.V_trim}/{rows}, best of 2"}
+    except Exception as ex:       # the one-thread figure is an extra; the all-cores figure above is the baseline
+        out["one_thread"] = {"value": None, "why": str(ex)[:200]}
+    return out
 
 
 def run_reference(args):
@@ -429,7 +574,10 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": round(us_full, 1), "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 4),
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD_NAME},
+            "config": bench_config(WORKLOAD_NAME, cold="host memory (the oracle reads its inputs from RAM)",
+                                   step="one oracle.draft_head call on a sample of the vocabulary rows, scaled",
+                                   launch="host function call", parallelism="host threads",
+                                   calls_per_s=round(1e6 / us_full, 3)),
             "cpu_baseline": {"value": round(us_full, 1), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                              "sample": f"each step runs the oracle on the first {rows} of {Vt} vocabulary rows "
                                        f"(all {M} draft rows); value scaled by {Vt}/{rows}"},

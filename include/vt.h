@@ -186,6 +186,16 @@ vt_status vt_coverage(const int32_t* token_ids, int64_t N,
                       uint64_t* covered_out, double* fraction_out,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same count (Eq. 2) in two steps, for callers that must not synchronise where the work is enqueued:
+ * vt_coverage_enqueue puts the bitmap build and the count on the stream and returns at once (same arguments and
+ * errors as vt_coverage, minus the outputs); vt_coverage_result SYNCHRONISES the stream and reads the count
+ * that the last enqueue on this workspace left in it (N = that call's N, for the fraction). */
+vt_status vt_coverage_enqueue(const int32_t* token_ids, int64_t N,
+                              const int32_t* keep_ids, int V_trim, int V_full,
+                              void* workspace, size_t workspace_bytes, void* stream);
+vt_status vt_coverage_result(void* workspace, int64_t N,
+                             uint64_t* covered_out, double* fraction_out, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Vocabulary-size selection (the paper's method, Sections 2.1-2.5), as an exhaustive scan over k:
  *

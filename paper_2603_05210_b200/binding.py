@@ -38,6 +38,8 @@ SYMBOLS = {
     "vt_draft_head_host": (_i, [_p, _p, _p, _i, _i, _i, _i, _p, _p, _p, _sz, _p]),
     "vt_last_status": (_i, [_p, _p]),
     "vt_coverage": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p, _sz, _p]),
+    "vt_coverage_enqueue": (_i, [_p, _i64, _p, _i, _i, _p, _sz, _p]),
+    "vt_coverage_result": (_i, [_p, _i64, _p, _p, _p]),
     "vt_select_workspace_bytes": (_sz, [_i]),
     "vt_select_vocab": (_i, [_p, _i64, _i, _i, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i, _i, _p, _p, _p, _p, _p,
                             _p, _p, _sz, _p]),
@@ -208,6 +210,22 @@ def vt_coverage(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int,
                              keep_ids.data_ptr(), keep_ids.numel(), V_full,
                              ctypes.addressof(covered), ctypes.addressof(frac),
                              workspace.data_ptr(), workspace.numel(), _stream()), "vt_coverage")
+    return int(covered.value), float(frac.value)
+
+
+def vt_coverage_enqueue(token_ids: torch.Tensor, keep_ids: torch.Tensor, V_full: int, workspace: torch.Tensor) -> None:
+    token_ids = _i32(token_ids, "token_ids")
+    keep_ids = _i32(keep_ids, "keep_ids")
+    _check(lib().vt_coverage_enqueue(token_ids.data_ptr() if token_ids.numel() else None, token_ids.numel(),
+                                     keep_ids.data_ptr(), keep_ids.numel(), V_full,
+                                     workspace.data_ptr(), workspace.numel(), _stream()), "vt_coverage_enqueue")
+
+
+def vt_coverage_result(workspace: torch.Tensor, N: int) -> tuple[int, float]:
+    covered = ctypes.c_uint64(0)
+    frac = ctypes.c_double(0.0)
+    _check(lib().vt_coverage_result(workspace.data_ptr(), int(N), ctypes.addressof(covered), ctypes.addressof(frac),
+                                    _stream()), "vt_coverage_result")
     return int(covered.value), float(frac.value)
 
 

@@ -64,8 +64,8 @@ static vt_status check_head_args(const void* h, const void* W, const int32_t* d2
     return VT_OK;
 }
 
-// Draft rows up to which the last head CTA merges the per-CTA records itself (one row per warp);
-// beyond that a separate merge kernel spreads the rows over many SMs.
+// Draft rows up to which a head kernel merges the per-CTA records itself (the warp that publishes a row last of
+// all CTAs merges it); beyond that the row-wise merge kernel spreads the rows over many SMs.
 constexpr int kFusedMergeMaxM = 16;
 
 static HeadOut make_out(const int32_t* d2t, int M, int Vt, int k, int32_t* tid, float* lp, int32_t* did, float* lse,
@@ -102,11 +102,12 @@ static bool auto_prefers_gemv(int M, int d, int Vt) {
 static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
     int grid = 0;
     vt_status r;
-    bool merged = c.out.fused_merge != 0;     // the vocabulary-rows-on-lanes kernel always merges row by row itself
+    bool merged = c.out.fused_merge != 0;     // the tensor-core kernels see to the merge themselves
     if (path == VT_PATH_GEMV) {
         r = launch_head_gemv(c, st, &grid);
     } else if (path == VT_PATH_MMA) {
         r = launch_head_mma(c, st, &grid);
+        merged = true;
     } else if (path == VT_PATH_MMA_SMALL) {
         r = launch_head_mma_small(c, st, &grid);
         merged = true;
@@ -118,10 +119,14 @@ static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
         merged = true;     // launched (or failed for a reason another path would not cure)
     } else {
         r = launch_head_mma(c, st, &grid);
-        if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) r = launch_head_gemv(c, st, &grid);
+        merged = true;
+        if (r == VT_ERR_UNSUPPORTED && gemv_supports(c.d)) {
+            r = launch_head_gemv(c, st, &grid);
+            merged = c.out.fused_merge != 0;
+        }
     }
     if (r != VT_OK) return r;
-    if (!merged) r = launch_merge(c.out, grid, st);
+    if (!merged) r = launch_merge_rowmajor(c.out, grid, st);
     return r;
 }
 
@@ -293,9 +298,8 @@ vt_status vt_last_status(void* workspace, void* stream) {
     return (status & kStatusTimeout) ? VT_ERR_TIMEOUT : VT_OK;
 }
 
-vt_status vt_coverage(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
-                      uint64_t* covered_out, double* fraction_out, void* workspace, size_t workspace_bytes,
-                      void* stream) {
+vt_status vt_coverage_enqueue(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
+                              void* workspace, size_t workspace_bytes, void* stream) {
     g_launches = 0;
     if (!keep_ids || (!token_ids && N > 0)) return VT_ERR_NULL;
     if (V_full < 1 || V_trim < 1 || N < 0) return VT_ERR_SHAPE;
@@ -306,14 +310,26 @@ vt_status vt_coverage(const int32_t* token_ids, int64_t N, const int32_t* keep_i
     cudaStream_t st = (cudaStream_t)stream;
     vt_status r = launch_keep_bitmap(keep_ids, V_trim, V_full, workspace, st);
     if (r != VT_OK) return r;
-    r = launch_coverage_count(token_ids, N, V_full, workspace, st);
-    if (r != VT_OK) return r;
+    return launch_coverage_count(token_ids, N, V_full, workspace, st);
+}
+
+vt_status vt_coverage_result(void* workspace, int64_t N, uint64_t* covered_out, double* fraction_out, void* stream) {
+    if (!workspace || !aligned(workspace, 256)) return VT_ERR_WORKSPACE;
+    if (N < 1) return VT_ERR_EMPTY;
     CoverageCounters c;
-    r = read_counters(workspace, st, &c);
+    vt_status r = read_counters(workspace, (cudaStream_t)stream, &c);
     if (r != VT_OK) return r;
     if (covered_out) *covered_out = c.covered;
     if (fraction_out) *fraction_out = (double)c.covered / (double)N;
     return VT_OK;
+}
+
+vt_status vt_coverage(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
+                      uint64_t* covered_out, double* fraction_out, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    vt_status r = vt_coverage_enqueue(token_ids, N, keep_ids, V_trim, V_full, workspace, workspace_bytes, stream);
+    if (r != VT_OK) return r;
+    return vt_coverage_result(workspace, N, covered_out, fraction_out, stream);
 }
 
 vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V_trim, float* logits, void* workspace,

@@ -168,7 +168,17 @@ __global__ void __launch_bounds__(kCoverageThreads) coverage_count_kernel(
     unsigned int c = 0;
     const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long gstride = (long long)gridDim.x * blockDim.x;
-    for (long long i = gtid; i < nvec; i += gstride) {
+    // four independent 16-byte loads per thread and trip keep enough bytes in flight to cover HBM latency
+    long long i = gtid;
+    for (; i + 3 * gstride < nvec; i += 4 * gstride) {
+        int4 t[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) t[u] = __ldcs(&vec[i + u * gstride]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            c += member(bm, t[u].x, V_full) + member(bm, t[u].y, V_full) + member(bm, t[u].z, V_full) + member(bm, t[u].w, V_full);
+    }
+    for (; i < nvec; i += gstride) {
         const int4 t = __ldcs(&vec[i]);
         c += member(bm, t.x, V_full) + member(bm, t.y, V_full) + member(bm, t.z, V_full) + member(bm, t.w, V_full);
     }
@@ -198,8 +208,8 @@ vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full,
     static std::atomic<unsigned long long> smem_configured{0};
     if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(coverage_count_kernel), (int)((int)kCoverageSmemBitmapMax), &smem_configured); rc != VT_OK)
         return rc;
-    const long long per_cta = (long long)kCoverageThreads * 4 * 8;   // ids one CTA takes in 8 trips
-    const int grid = (int)std::max(1LL, std::min((N + per_cta - 1) / per_cta, (long long)sms * 2));
+    const long long per_cta = (long long)kCoverageThreads * 4 * 8;   // ids one CTA takes in two trips of four loads
+    const int grid = (int)std::max(1LL, std::min((N + per_cta - 1) / per_cta, (long long)sms * 4));
     coverage_count_kernel<<<grid, kCoverageThreads, smem, st>>>(token_ids, N, V_full, bitmap, (int)words, in_smem,
                                                                counters);
     count_launch();

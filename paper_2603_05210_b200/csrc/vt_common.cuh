@@ -1,6 +1,6 @@
 // Shared device/host helpers of the draft-head library: workspace layout, PTX wrappers for
-// mbarriers and bulk copies with bounded waits, sortable (logit, index) keys, the per-thread
-// top-k list and the cross-CTA merge that ends a draft-head call.
+// mbarriers and bulk copies with bounded waits, sortable (logit, index) keys, the per-warp and per-thread
+// top-k updates and the cross-CTA merge that ends a draft-head call.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -12,14 +12,12 @@ namespace vt {
 
 // ------------------------------------------------------------------------------------------
 // Workspace of a draft-head call:
-//   [0, 512)                          WsHeader
-//   recs [kMaxParts][pitch] u64       per-CTA partial results: M records of KS slots, then padding
-//                                     slots 0..k-1  top-k list as sortable keys, descending, 0-padded
-//                                     slot  k       (running max, sum of exp(x - max)) as two floats
-//                                     KS = k + 1 rounded up to even, so every record is 16-byte aligned;
-//                                     pitch = M * KS, plus 2 when that makes pitch / 2 odd: all CTAs' records
-//                                     can then be copied to shared memory as one block and read there by 32
-//                                     lanes (one CTA each) with at most 2-way bank conflicts
+//   [0, 512)   WsHeader
+//   records    per draft row m, kMaxParts * (k + 1) consecutive u64 (row-major: what one CTA wrote for one row is
+//              strided, what all CTAs wrote for one row is contiguous, so the warp that merges a row reads every
+//              CTA's j-th best key with one coalesced load):
+//                ms   [kMaxParts]        every CTA's (running max, sum of exp(x - max)) as two floats
+//                keys [k][kMaxParts]     keys[j][p] = CTA p's j-th best candidate as a sortable key, 0 = none
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxParts = 256;             // upper bound on CTAs that contribute partials
 constexpr size_t kHeaderBytes = 512;
@@ -27,7 +25,7 @@ constexpr size_t kHeaderBytes = 512;
 constexpr int kRowTickets = 64;            // draft rows that can be merged row by row (one ticket each)
 
 struct WsHeader {
-    unsigned int ticket;     // CTAs that have published their partials in the running call
+    unsigned int reserved;
     unsigned int status;     // bit 0: a bounded wait ran out
     unsigned int row_ticket[kRowTickets];   // per draft row: CTAs that have published that row (row-wise merge)
     unsigned int pad[126 - kRowTickets];
@@ -36,24 +34,11 @@ static_assert(sizeof(WsHeader) == kHeaderBytes, "header is two 256-byte lines");
 
 constexpr unsigned int kStatusTimeout = 1u;
 
-__host__ __device__ inline int ws_slots(int k) { return (k + 2) & ~1; }
-__host__ __device__ inline int ws_pitch(int M, int k) {
-    const int raw = M * ws_slots(k);
-    return ((raw >> 1) & 1) ? raw : raw + 2;
-}
 __host__ __device__ inline size_t ws_total_bytes(int M, int k) {
-    size_t b = kHeaderBytes + (size_t)kMaxParts * ws_pitch(M, k) * 8;
+    size_t b = kHeaderBytes + (size_t)M * kMaxParts * (size_t)(k + 1) * 8;
     return (b + 255) & ~(size_t)255;
 }
 
-// Record of (CTA p, draft row m).
-#define VT_REC(o, p, m) ((o).recs + (size_t)(p) * ws_pitch((o).M, (o).k) + (size_t)(m) * ws_slots((o).k))
-
-// Row-major records (the row-wise merge of the few-draft-rows kernel): draft row m owns kMaxParts * (k + 1)
-// consecutive u64 of the same record area,
-//   ms   [kMaxParts]        every CTA's (max, sum-exp)
-//   keys [k][kMaxParts]     keys[j][p] = CTA p's j-th best key: one coalesced read per depth
-// M * kMaxParts * (k + 1) <= kMaxParts * ws_pitch(M, k), so the area vt_workspace_bytes sizes holds either layout.
 #define VT_ROW_MS(o, m) ((o).recs + (size_t)(m) * kMaxParts * ((o).k + 1))
 #define VT_ROW_KEYS(o, m, j) (VT_ROW_MS(o, m) + (size_t)((j) + 1) * kMaxParts)
 
@@ -68,7 +53,7 @@ struct HeadOut {
     WsHeader* hdr;
     unsigned long long* recs;
     int M, k, Vt;
-    int fused_merge;      // 1: the last CTA to publish merges; 0: a merge kernel follows
+    int fused_merge;      // 1: the warp that publishes a row last of all CTAs merges it; 0: the merge kernel follows
 };
 
 #ifdef __CUDACC__
@@ -205,6 +190,47 @@ __device__ __forceinline__ unsigned long long pack_ms(float mx, float s) {
 __device__ __forceinline__ float2 unpack_ms(unsigned long long v) {
     return make_float2(__uint_as_float((uint32_t)v), __uint_as_float((uint32_t)(v >> 32)));
 }
+
+
+// ------------------------------------------------------------------------------------------
+// Thread-private top-k: one thread owns one draft row and keeps its KR best (logit, index) pairs in registers.
+// ------------------------------------------------------------------------------------------
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sorted insertion into a thread's register list: v descends, equal logits keep their order of arrival (logits
+// reach a thread in ascending vocabulary order, so a later equal one ranks below).  p[j] = "x beats entry j" is
+// monotone in j; entry j takes its upper neighbour where that one is beaten, x where only it is, else stays.
+// Inserting a logit that beats nothing changes nothing.
+template <int KR>
+__device__ __forceinline__ void rows_insert(float (&v)[KR], int (&ix)[KR], float x, int xi) {
+    bool p[KR];
+#pragma unroll
+    for (int j = 0; j < KR; ++j) p[j] = x > v[j];
+#pragma unroll
+    for (int j = KR - 1; j > 0; --j) {
+        v[j] = p[j - 1] ? v[j - 1] : (p[j] ? x : v[j]);
+        ix[j] = p[j - 1] ? ix[j - 1] : (p[j] ? xi : ix[j]);
+    }
+    v[0] = p[0] ? x : v[0];
+    ix[0] = p[0] ? xi : ix[0];
+}
+
+// The same insertion for logits alone (no indices): two min/max per entry.
+template <int KR>
+__device__ __forceinline__ void vals_insert(float (&g)[KR], float x) {
+#pragma unroll
+    for (int j = KR - 1; j > 0; --j) g[j] = fmaxf(g[j], fminf(g[j - 1], x));
+    g[0] = fmaxf(g[0], x);
+}
+
+// Register-list length for a top-k of k: the smallest instantiated length that holds k entries, 0 if none does.
+__host__ __device__ inline int topk_list_regs(int k) { return k <= 4 ? 4 : k <= 8 ? 8 : k <= 10 ? 10 : k <= 16 ? 16 : 0; }
 
 // Warp-wide maximum of 64-bit keys with two 32-bit redux operations.
 __device__ __forceinline__ unsigned long long warp_max_key(unsigned long long v) {
@@ -436,18 +462,6 @@ __device__ __forceinline__ void write_winner(const HeadOut& o, int m, int j, uns
     }
 }
 
-// Final merge of one draft row: writes its k winners (descending), their log-probs and target ids.
-// Winners are written by the lanes that hold them, so the d2t gathers are one round trip, not k.
-__device__ inline void merge_row_final(const HeadOut& o, int P, int m, const unsigned long long* rec, int stride,
-                                       unsigned long long* cbuf) {
-    const int lane = threadIdx.x & 31;
-    const int k = o.k;
-    const float2 ms = warp_merge_ms(rec, stride, P, k);
-    const float lse = ms.x + __logf(ms.y);
-    warp_select_topk(rec, stride, P, k, cbuf, [&](int j, unsigned long long best) { write_winner(o, m, j, best, lse); });
-    if (lane == 0 && o.lse) o.lse[m] = lse;
-}
-
 // Row-wise final merge by one warp, straight from the row-major records in global memory (VT_ROW_*), for the
 // warp that published draft row m last.  One round trip to L2 brings every CTA's (max, sum-exp) and its three
 // best keys into registers (lane L owns CTAs L, L+32, ...); the log-sum-exp follows from the former.  Every list
@@ -518,81 +532,6 @@ __device__ inline void merge_row_global(const HeadOut& o, int P, int m) {
     else merge_row_global_n<kMergeSlots>(o, P, m);
 }
 
-// Publishes this CTA's records (already written to global memory by the calling threads) and
-// returns true in every thread of the last CTA to arrive.  Must be called by all threads.
-__device__ inline bool publish_and_check_last(WsHeader* hdr, int* smem_flag) {
-    __threadfence();
-    fence_proxy_async();          // the merging CTA reads the records with bulk copies (async proxy)
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int t = atomicAdd(&hdr->ticket, 1u);
-        *smem_flag = (t == gridDim.x - 1) ? 1 : 0;
-        __threadfence();
-    }
-    __syncthreads();
-    return *smem_flag != 0;
-}
-
-// Merges draft rows [m_begin, m_begin + m_count) from the records of P CTAs.  The records of a batch
-// of rows are brought into shared memory with one bulk copy per CTA record block (P copies in
-// flight at once: one L2 round trip per batch), then each warp merges one row at a time.
-//   stage_base/stage_bytes: shared memory the CTA no longer uses, 16-byte aligned, at least
-//                           P * (KS * 8 + 16) + (warps of the CTA) * 2048 bytes;
-//   bar: an initialised mbarrier (count 1), phase 0.
-// Must be called by all threads of the CTA.
-__device__ inline void merge_rows(const HeadOut& o, int P, int m_begin, int m_count,
-                                  unsigned char* stage_base, size_t stage_bytes, uint32_t bar) {
-    const int warp = threadIdx.x >> 5;
-    const int nwarps = blockDim.x >> 5;
-    const int KS = ws_slots(o.k), M = o.M;
-    // the tail of the region holds one candidate buffer per warp (warp_select_topk)
-    const size_t cand_bytes = (size_t)nwarps * kMergeCand * 8;
-    unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(stage_base + stage_bytes - cand_bytes) +
-                               (size_t)warp * kMergeCand;
-    stage_bytes -= cand_bytes;
-    const int pitch = ws_pitch(M, o.k);
-    unsigned long long* stage = reinterpret_cast<unsigned long long*>(stage_base);
-    const size_t all_bytes = (size_t)P * pitch * 8;
-    const bool one_copy = m_begin == 0 && m_count == M && all_bytes <= stage_bytes && all_bytes < (1u << 20);
-    int batch = one_copy ? m_count : (int)((stage_bytes / P - 16) / ((size_t)KS * 8));
-    const int tx_cap = (int)(((1u << 20) - 16) / ((size_t)P * KS * 8));     // mbarrier byte-count limit
-    if (!one_copy && batch > tx_cap) batch = tx_cap;
-    if (batch > m_count) batch = m_count;
-    if (batch < 1) batch = 1;
-    fence_proxy_async();          // shared memory last touched by ordinary loads/stores is reused by bulk copies
-    __syncthreads();
-    uint32_t phase = 0;
-    for (int b0 = 0; b0 < m_count; b0 += batch, phase ^= 1u) {
-        const int nb = min(batch, m_count - b0);
-        int stride;                                            // u64 units between CTA record blocks in shared memory
-        if (one_copy) {
-            // every CTA's records for all rows, padding included, are one contiguous block: a single copy
-            stride = pitch;
-            if (threadIdx.x == 0) {
-                mbar_arrive_expect_tx(bar, (uint32_t)all_bytes);
-                bulk_g2s(smem_u32(stage), o.recs, (uint32_t)all_bytes, bar);
-            }
-        } else {
-            stride = nb * KS;
-            if (((stride >> 1) & 1) == 0) stride += 2;         // odd multiple of 16 bytes: at most 2-way bank conflicts
-            const uint32_t bytes = (uint32_t)nb * KS * 8;
-            // The phase needs thread 0's arrival as well as all the bytes, so copies that land before the
-            // byte count is posted cannot complete it early: no barrier between posting and issuing.
-            if (threadIdx.x == 0) mbar_arrive_expect_tx(bar, bytes * (uint32_t)P);
-            for (int p = threadIdx.x; p < P; p += blockDim.x)
-                bulk_g2s(smem_u32(stage + (size_t)p * stride), VT_REC(o, p, m_begin + b0), bytes, bar);
-        }
-        // every thread takes the same decision, so none is left alone at the barrier that ends the batch
-        const bool timed_out = !mbar_wait(bar, phase);
-        if (__syncthreads_or(timed_out ? 1 : 0)) {
-            if (timed_out) atomicOr(&o.hdr->status, kStatusTimeout);
-            break;
-        }
-        for (int r = warp; r < nb; r += nwarps)
-            merge_row_final(o, P, m_begin + b0 + r, stage + (size_t)r * KS, stride, cbuf);
-        __syncthreads();
-    }
-}
 #endif  // __CUDACC__
 
 }  // namespace vt

@@ -9,8 +9,8 @@
 // packed fp32x2 FMAs, and fold the lane partials with a transposing shuffle reduction.  The lane
 // that ends up with a logit keeps that (row slot, draft row)'s running (max, sum-exp) and top-k
 // list, so no logit is written to memory and no warp waits for another.  When the range is done
-// the CTA folds its warps' lists into one record per draft row; the last CTA to publish merges all
-// CTAs' records (or a merge kernel does, for many draft rows).
+// the CTA folds its warps' lists into one record per draft row; the warp that publishes a row last of all
+// CTAs merges it (or the row-wise merge kernel does, for many draft rows).
 //
 // The FP32 pipe bounds this path: every weight costs M fused multiply-adds, which the CUDA cores
 // keep up with only for M <= 4; larger M belongs to the tensor-core path.
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
     const int nrows = row_end - row_begin;
     const int SR = p.rows_per_stage, S = p.n_stages;
     const int ntiles = (nrows + SR - 1) / SR;
-    const int KS = ws_slots(k);
+    const int KS = ((k + 2) & ~1);
 
     unsigned char* hs = smem + p.h_off;                                                      // [MP][d] bf16
     unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [consumer][NV][KS]
@@ -232,13 +232,14 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         const int stride = MP * KS;
         const float2 ms = warp_merge_ms(rec0, stride, P1, k);
         unsigned long long* cbuf = reinterpret_cast<unsigned long long*>(smem + p.fold_off) + (size_t)warp * kMergeCand;
+        // Row-major record; with few draft rows then the row's ticket: the warp that draws the last one (over all
+        // CTAs) merges the row at once, straight from global memory, with no CTA-wide step between the fold and
+        // the outputs.  With many draft rows the row-wise merge kernel follows instead.
+        const int row = p.m_begin + m;
+        warp_select_topk(rec0, stride, P1, k, cbuf,
+                         [&](int j, unsigned long long best) { VT_ROW_KEYS(p.out, row, j)[cta] = best; });
+        if (lane == 0) VT_ROW_MS(p.out, row)[cta] = pack_ms(ms.x, ms.y);
         if (p.out.fused_merge) {
-            // Row-major record, then the row's ticket: the warp that draws the last one (over all CTAs) merges the
-            // row at once, straight from global memory.  No CTA-wide step between the fold and the outputs.
-            const int row = p.m_begin + m;
-            warp_select_topk(rec0, stride, P1, k, cbuf,
-                             [&](int j, unsigned long long best) { VT_ROW_KEYS(p.out, row, j)[cta] = best; });
-            if (lane == 0) VT_ROW_MS(p.out, row)[cta] = pack_ms(ms.x, ms.y);
             __threadfence();
             __syncwarp();
             unsigned int ticket = 0;
@@ -249,10 +250,6 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
                 merge_row_global(p.out, G, row);
                 if (lane == 0) p.out.hdr->row_ticket[row] = 0u;        // ready for the next call
             }
-        } else {
-            unsigned long long* dst = VT_REC(p.out, cta, p.m_begin + m);
-            warp_select_topk(rec0, stride, P1, k, cbuf, [&](int j, unsigned long long best) { dst[j] = best; });
-            if (lane == 0) dst[k] = pack_ms(ms.x, ms.y);
         }
     }
 }
@@ -281,7 +278,7 @@ vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid_out) {
     if (rs != VT_OK) return rs;
     const int grid = head_grid(sms, c.Vt);
     *grid_out = grid;
-    const int KS = ws_slots(c.out.k);
+    const int KS = ((c.out.k + 2) & ~1);
 
     for (int m0 = 0; m0 < c.M; m0 += kGemvMaxM) {
         const int mc = std::min(kGemvMaxM, c.M - m0);

@@ -52,7 +52,9 @@ struct SmallParams {
     int M;                    // draft rows of this launch, <= kSmMaxM
     int m_begin;              // first of them among the call's draft rows
     int merge_in_kernel;      // 1: one draft row per epilogue warp, merged by the last warp to publish it; 0: a merge kernel follows
-    int n_epi;                // epilogue warps: 8, or 16 when M > 8; the block has two more (producer, MMA issuer)
+    int n_epi;                // epilogue warps: 8, or 16 when M > 8 with the warp-per-row epilogue; the block has
+                              // two more (producer, MMA issuer)
+    int lg_rows;              // draft rows whose tile logits shared memory holds at a time: kLgRows, or all with thread-per-row
     uint32_t scratch_stride;  // bytes of one epilogue warp's candidate buffer: (128 + k) keys
     int N;                    // MMA N: M rounded up to a multiple of 16
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
@@ -95,6 +97,9 @@ __device__ __forceinline__ void reader_barrier() { asm volatile("bar.sync 2, 128
 // Barrier among the epilogue warps only (the producer and the MMA issuer never join it).
 __device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); }
 
+// KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue for more than 16 draft rows, with a
+// register list of KR >= k entries per thread.
+template <int KR>
 __global__ void __launch_bounds__(kSmThreads, 1)
 head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
                       const SmallParams p) {
@@ -142,10 +147,12 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         *abort_flag = 0;
         fence_mbar_init();
     }
-    for (int i = tid; i < M * k; i += blockDim.x) lists[i] = 0ull;
-    if (tid < kSmMaxM) {
-        ms_s[tid] = make_float2(-INFINITY, 0.0f);
-        tau_s[tid] = -INFINITY;
+    if (KR == 0) {
+        for (int i = tid; i < M * k; i += blockDim.x) lists[i] = 0ull;
+        if (tid < kSmMaxM) {
+            ms_s[tid] = make_float2(-INFINITY, 0.0f);
+            tau_s[tid] = -INFINITY;
+        }
     }
     // With 8 rows of h per k-block the MMA's rows 8-15 alias whatever follows the block (the next k-block of a
     // resident h, the next ring slot otherwise): accumulator columns nobody reads.  After the last block of a
@@ -276,7 +283,261 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 (void)mbar_wait(bar_drain, 0u);
             }
         }
-    } else if (warp < p.n_epi) {
+    } else if (KR > 0 && warp < p.n_epi) {
+        // ------------------------------------------------------------------ epilogue, one draft row per thread
+        // Warps 0-3 read a finished tile out of TMEM (lane = vocabulary row, 16 draft rows per load) and lay it
+        // out per draft row in shared memory.  Then each of their threads owns ONE draft row (and, with fewer than
+        // 128 draft rows, one of several column ranges of it) and scans its logits alone, keeping a sorted list
+        // of the KR best (logit, index) pairs in registers - no shuffle, no ballot, no barrier between threads.
+        // A row's first scan bounds the candidates first: the KR-th largest of the maxima of groups of 4 or 8
+        // logits has at least KR logits at or above it, so nothing below it can be among the KR best; the few
+        // logits that pass are marked in a bit mask and inserted one per turn of a loop that runs for the busiest
+        // lane's count.  Later tiles are filtered by the list's own last entry.  Warps 4-7 mirror that thread
+        // assignment and fold the same logits into the rows' running (max, sum-exp): the two kinds of work use
+        // different pipes (compare/select against multiply-add and exp2) and hide each other's latencies.
+        constexpr int KL = KR > 0 ? KR : 1;
+        const bool scanner = warp < 4;
+        const int w4 = warp & 3;
+        const int RG = (M + 31) >> 5;                                  // groups of 32 draft rows: 1 .. 4
+        const int Q = RG == 1 ? 4 : RG == 2 ? 2 : 1;                   // column ranges a row is split into
+        const int rg = w4 % RG, part = w4 / RG;
+        const bool works = part < Q;                                   // warp-uniform
+        const int m_own = rg * 32 + lane;                              // the thread's draft row of this pass
+        const int xs = RG * 32;
+        const float* rowp = lg + (size_t)min(m_own, M - 1) * kLgPitch;     // lanes past the last row re-read it and keep nothing
+        float v[KL];
+        int ix[KL];
+#pragma unroll
+        for (int j = 0; j < KL; ++j) { v[j] = -INFINITY; ix[j] = -1; }
+        float mx = -INFINITY, ssum = 0.0f;
+        int seen = 0;                                                  // logits this thread has scanned (the same in every lane of a warp)
+        for (int t = 0; t < ntiles; ++t) {
+            const int buf = t & 1;
+            const int row0 = row_begin + t * TH;
+            const int nv = min(TH, row_end - row0);
+            if (scanner) {
+                // warp-uniform decisions: tcgen05.ld needs the whole warp
+                bool got = false;
+                if (!__any_sync(0xFFFFFFFFu, *abort_flag != 0)) {
+                    got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u));
+                    if (!got) fail();
+                }
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
+                if (KF > 1) {
+                    // Folded k-blocks: this warp's lanes are k-group g of tile rows r0 + lane, and columns
+                    // NG*g .. NG*g + NG - 1 of the accumulator are their partial logits for the draft rows.
+                    const int SR = 128 / KF, NG = p.NG, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
+                    float* partial = reinterpret_cast<float*>(smem + p.part_off);
+                    if (got) {
+                        tc_fence_after();
+                        for (int c0 = 0; c0 < NG; c0 += 16) {
+                            uint32_t u[16];
+                            tc_ld16(taddr + (uint32_t)(NG * g + c0), u);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int m = 0; m < 16; ++m) partial[(g * NG + c0 + m) * 64 + r] = __uint_as_float(u[m]);
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+                    }
+                    reader_barrier();                              // all four readers' partial sums are in place
+                    for (int e = tid; e < M * SR; e += 128) {
+                        const int m = e / SR, rr = e - m * SR;
+                        if (rr >= nv) continue;
+                        float sum = 0.0f;
+                        for (int gg = 0; gg < KF; ++gg) sum += partial[(gg * p.NG + m) * 64 + rr];
+                        lg[m * kLgPitch + rr] = sum;
+                        if (p.out.logits) p.out.logits[(size_t)(p.m_begin + m) * Vt + row0 + rr] = sum;
+                    }
+                } else if (got) {
+                    const int i = warp * 32 + lane;                // TMEM lane = vocabulary row of the tile
+                    tc_fence_after();
+                    for (int c1 = 0; c1 < M; c1 += 16) {           // 16 draft rows per load
+                        uint32_t u[16];
+                        tc_ld16(taddr + (uint32_t)c1, u);
+                        tc_wait_ld();
+                        if (i < nv) {
+#pragma unroll
+                            for (int m = 0; m < 16; ++m)
+                                if (c1 + m < M) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(u[m]);
+                            if (p.out.logits) {
+#pragma unroll
+                                for (int m = 0; m < 16; ++m)
+                                    if (c1 + m < M)
+                                        p.out.logits[(size_t)(p.m_begin + c1 + m) * Vt + row0 + i] = __uint_as_float(u[m]);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                }
+            }
+            epi_barrier(256);                                      // the tile's logits are in shared memory
+            // ---- the thread's own columns [cb, ce) of its draft row.  After a wait ran out the buffer holds the
+            // previous tile again: whatever is computed from it belongs to a call that reports the time-out.
+            const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
+            const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
+            const int nch = (n + 15) >> 4;
+            auto load16 = [&](int q, float (&x)[16]) {             // chunk q of the range, columns past it as -inf
+                const int c = cb + 16 * q;
+#pragma unroll
+                for (int u4 = 0; u4 < 4; ++u4) {
+                    const float4 f = *reinterpret_cast<const float4*>(rowp + c + 4 * u4);
+                    x[4 * u4 + 0] = f.x; x[4 * u4 + 1] = f.y; x[4 * u4 + 2] = f.z; x[4 * u4 + 3] = f.w;
+                }
+                const int left = ce - c;
+                if (left < 16) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) x[e] = e < left ? x[e] : -INFINITY;
+                }
+            };
+            if (works && n > 0 && !scanner) {
+                // running log-sum-exp of the row over these columns: (max, sum of exp(x - max))
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (q < nch) {
+                        float x[16];
+                        load16(q, x);
+                        float cm = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+                        cm = fmaxf(cm, fmaxf(fmaxf(fmaxf(x[8], x[9]), fmaxf(x[10], x[11])), fmaxf(fmaxf(x[12], x[13]), fmaxf(x[14], x[15]))));
+                        const float nm = fmaxf(mx, cm);
+                        const float nml = nm * kLog2e;
+                        float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+                        for (int e = 0; e < 16; e += 2) {
+                            a0 += ex2_approx(fmaf(x[e], kLog2e, -nml));             // exp(-inf) = 0
+                            a1 += ex2_approx(fmaf(x[e + 1], kLog2e, -nml));
+                        }
+                        ssum = ssum * ex2_approx((mx - nm) * kLog2e) + (a0 + a1);   // first chunk: 0 * 0
+                        mx = nm;
+                    }
+                }
+            }
+            if (works && n > 0 && scanner) {
+                const bool full = seen >= KL;
+                const int gs = full ? 0 : n >= 8 * (KL + 2) ? 8 : n >= 4 * (KL + 2) ? 4 : 0;
+                if (!full && gs == 0) {
+                    // a short first range: every logit goes through the list
+                    for (int q = 0; q < nch; ++q) {
+                        float x[16];
+                        load16(q, x);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) rows_insert<KL>(v, ix, x[e], row0 + cb + 16 * q + e);
+                    }
+                } else {
+                    float tau = v[KL - 1];
+                    if (!full) {       // bound from group maxima: at least KL + 2 whole groups exist
+                        float g[KL];
+#pragma unroll
+                        for (int j = 0; j < KL; ++j) g[j] = -INFINITY;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            if (q < nch) {
+                                float x[16];
+                                load16(q, x);
+                                if (gs == 8) {
+#pragma unroll
+                                    for (int u8 = 0; u8 < 2; ++u8)
+                                        vals_insert<KL>(g, fmaxf(fmaxf(fmaxf(x[8 * u8], x[8 * u8 + 1]), fmaxf(x[8 * u8 + 2], x[8 * u8 + 3])),
+                                                                 fmaxf(fmaxf(x[8 * u8 + 4], x[8 * u8 + 5]), fmaxf(x[8 * u8 + 6], x[8 * u8 + 7]))));
+                                } else {
+#pragma unroll
+                                    for (int u4 = 0; u4 < 4; ++u4)
+                                        vals_insert<KL>(g, fmaxf(fmaxf(x[4 * u4], x[4 * u4 + 1]), fmaxf(x[4 * u4 + 2], x[4 * u4 + 3])));
+                                }
+                            }
+                        }
+                        tau = g[KL - 1];
+                    }
+                    // candidates: above the list's last entry (a later row loses a tie), or not below the bound
+                    uint32_t mk[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (q < nch) {
+                            float x[16];
+                            load16(q, x);
+                            uint32_t bits = 0;
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) bits |= (full ? x[e] > tau : x[e] >= tau) ? (1u << e) : 0u;
+                            mk[q >> 1] |= bits << (16 * (q & 1));
+                        }
+                    }
+                    // one candidate per lane and turn; the next one's logit is fetched while this one is inserted
+                    auto next = [&](float& xv, int& xi) {
+                        xv = -INFINITY;
+                        xi = 0;
+                        const int w = mk[0] ? 0 : mk[1] ? 1 : mk[2] ? 2 : 3;
+                        const uint32_t word = w == 0 ? mk[0] : w == 1 ? mk[1] : w == 2 ? mk[2] : mk[3];
+                        if (word != 0u) {
+                            const int c = cb + 32 * w + __ffs(word) - 1;
+                            const uint32_t rest = word & (word - 1u);
+                            mk[0] = w == 0 ? rest : mk[0];
+                            mk[1] = w == 1 ? rest : mk[1];
+                            mk[2] = w == 2 ? rest : mk[2];
+                            mk[3] = w == 3 ? rest : mk[3];
+                            xv = rowp[c];
+                            xi = row0 + c;
+                        }
+                    };
+                    bool more = __any_sync(0xFFFFFFFFu, (mk[0] | mk[1] | mk[2] | mk[3]) != 0u);
+                    float nxv;
+                    int nxi;
+                    next(nxv, nxi);
+                    while (more) {
+                        const float xv = nxv;
+                        const int xi = nxi;
+                        more = __any_sync(0xFFFFFFFFu, (mk[0] | mk[1] | mk[2] | mk[3]) != 0u);
+                        next(nxv, nxi);
+                        rows_insert<KL>(v, ix, xv, xi);            // -inf beats nothing
+                    }
+                }
+            }
+            seen += max(n, 0);
+            epi_barrier(256);                                      // the buffer may be overwritten
+        }
+        // ---- the rows' records: best k keys and (max, sum-exp).  The logits buffer is free now: it takes every
+        // thread's list (or sums); the range-0 scanner of a row merges its column ranges and writes the record.
+        unsigned long long* xl = reinterpret_cast<unsigned long long*>(lg);      // [(part * RG * 32 + row) * (KL + 1)]
+        if (works) {
+            unsigned long long* mine = xl + (size_t)(part * xs + m_own) * (KL + 1);
+            if (scanner) {
+#pragma unroll
+                for (int j = 0; j < KL; ++j) mine[j] = ix[j] >= 0 ? make_key(v[j], ix[j]) : 0ull;
+            } else {
+                mine[KL] = pack_ms(mx, ssum);
+            }
+        }
+        epi_barrier(256);
+        if (scanner && part == 0 && m_own < M) {
+            const int row = p.m_begin + m_own;                                 // among the call's draft rows
+            // Q sorted lists: the best remaining key is the largest head, k times
+            int pos[4] = {0, 0, 0, 0};
+            for (int j = 0; j < k; ++j) {
+                unsigned long long best = 0ull;
+                int bq = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (q < Q && pos[q] < KL) {
+                        const unsigned long long key = xl[(size_t)(q * xs + m_own) * (KL + 1) + pos[q]];
+                        if (key > best) { best = key; bq = q; }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) pos[q] += (q == bq && best != 0ull) ? 1 : 0;
+                VT_ROW_KEYS(p.out, row, j)[cta] = best;
+            }
+            float cmx = -INFINITY;
+            for (int q = 0; q < Q; ++q) cmx = fmaxf(cmx, unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]).x);
+            float cs = 0.0f;
+            for (int q = 0; q < Q; ++q) {
+                const float2 ms = unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]);
+                if (ms.y > 0.0f) cs += ms.y * __expf(ms.x - cmx);
+            }
+            VT_ROW_MS(p.out, row)[cta] = pack_ms(cmx, cs);
+        }
+    } else if (KR == 0 && warp < p.n_epi) {
         // ------------------------------------------------------------------ epilogue warps
         const int n_epi = p.n_epi;
         if (warp == n_epi - 1 && lane == 0 && ntiles > 0 && p.h_resident) {
@@ -424,22 +685,30 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 
 // ------------------------------------------------------------------------------------------ host
 // Tile geometry and shared-memory layout for a shape; false if it does not fit.
-static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
+static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, int* list_regs) {
     if (M < 1 || M > kSmMaxM) return false;
     const int R = (Vt + grid - 1) / grid;                    // most rows a CTA owns
     const int nt = (R + 127) / 128;
+    // More than 16 draft rows: one thread per draft row, as long as a register list holds k entries.  With four
+    // and more tiles per CTA and at most 64 draft rows the warp-per-row epilogue hides behind the stream as well
+    // and leaves more shared memory to the ring (measured at V_trim = 128256: 180 against 194 us).
+    const int KR = (M > 16 && !(M <= 64 && nt >= 4)) ? topk_list_regs(k) : 0;
+    *list_regs = KR;
     p->M = M;
     p->d = d;
     p->nk = (d + kBoxK - 1) / kBoxK;
     p->TH = (R + nt - 1) / nt;
     p->w_tx = (uint32_t)p->TH * 128u;
     p->h_blk = M <= 8 ? 1024u : (uint32_t)(((M + 15) / 16) * 16) * 128u;
-    const size_t lg_bytes = ((size_t)std::min(M, kLgRows) * kLgPitch * 4 + 127) & ~(size_t)127;
-    const size_t list_bytes = (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
-    p->n_epi = M > 8 ? kSmMaxEpiWarps : 8;
-    p->merge_in_kernel = M <= p->n_epi;
+    p->lg_rows = KR > 0 ? ((M + 15) / 16) * 16 : std::min(M, kLgRows);
+    // thread-per-row: all of the tile's draft rows at once, and room for the column ranges' lists at the end
+    const size_t lg_bytes = KR > 0 ? (std::max((size_t)p->lg_rows * kLgPitch * 4, (size_t)128 * (KR + 1) * 8) + 127) & ~(size_t)127
+                                   : ((size_t)p->lg_rows * kLgPitch * 4 + 127) & ~(size_t)127;
+    const size_t list_bytes = KR > 0 ? 0 : (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
+    p->n_epi = KR > 0 ? 8 : M > 8 ? kSmMaxEpiWarps : 8;
+    p->merge_in_kernel = KR == 0 && M <= p->n_epi;
     p->scratch_stride = (uint32_t)(kSmCand - VT_MAX_K + k) * 8u;
-    const size_t scratch_bytes = ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
+    const size_t scratch_bytes = KR > 0 ? 0 : ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
     const size_t bar_bytes = (size_t)(2 * kSmMaxStages + 4 + kHParts + 1) * 8 + 16;
     const size_t common = 1024 + lg_bytes + list_bytes + scratch_bytes + bar_bytes + 128;
     // h resident only for M <= 8 (8 rows per k-block) and short tiles, where little is streamed and the fold by two
@@ -499,6 +768,18 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p) {
     return false;
 }
 
+template <int KR>
+static vt_status launch_small(const CUtensorMap& tmW, const CUtensorMap& tmH, const SmallParams& p, int grid, cudaStream_t st) {
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel<KR>), kMaxDynSmem, &smem_configured);
+        rc != VT_OK)
+        return rc;
+    cudaError_t e = launch_pdl(head_mma_small_kernel<KR>, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
+    count_launch();
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_out) {
     int sms = 0;
     vt_status r = device_sm_count(&sms);
@@ -506,17 +787,15 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
     // every pass of kSmMaxM draft rows must fit before anything is launched
+    int KR = 0;
     for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {
         SmallParams q{};
-        if (!small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &q)) return VT_ERR_UNSUPPORTED;
+        if (!small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &q, &KR)) return VT_ERR_UNSUPPORTED;
     }
-    static std::atomic<unsigned long long> smem_configured{0};
-    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel), (int)(kMaxDynSmem), &smem_configured); rc != VT_OK)
-        return rc;
     bool merge_after = false;
     for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {        // each pass streams the weights once for its draft rows
         SmallParams p{};
-        small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p);
+        small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p, &KR);
         p.out = c.out;
         p.m_begin = m0;
         p.early_weights = c.static_weights;
@@ -527,10 +806,14 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
         if (r != VT_OK) return r;
         r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
         if (r != VT_OK) return r;
-        cudaError_t e = launch_pdl(head_mma_small_kernel, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
-        count_launch();
-        if (e == cudaSuccess) e = cudaGetLastError();
-        if (e != cudaSuccess) return cuda_fail(e);
+        switch (KR) {
+            case 4: r = launch_small<4>(tmW, tmH, p, grid, st); break;
+            case 8: r = launch_small<8>(tmW, tmH, p, grid, st); break;
+            case 10: r = launch_small<10>(tmW, tmH, p, grid, st); break;
+            case 16: r = launch_small<16>(tmW, tmH, p, grid, st); break;
+            default: r = launch_small<0>(tmW, tmH, p, grid, st); break;
+        }
+        if (r != VT_OK) return r;
     }
     return merge_after ? launch_merge_rowmajor(c.out, grid, st) : VT_OK;
 }

@@ -59,8 +59,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid);
 // arrival ticket per draft row), everything else launches the row-wise merge kernel after itself;
 // VT_ERR_UNSUPPORTED when the shape does not fit
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid);
-vt_status launch_merge(const HeadOut& o, int P, cudaStream_t st);
-vt_status launch_merge_rowmajor(const HeadOut& o, int P, cudaStream_t st);   // records of launch_head_mma_small, M > 16
+vt_status launch_merge_rowmajor(const HeadOut& o, int P, cudaStream_t st);   // one warp per draft row over the row-major records
 
 vt_status launch_compact(const void* W_full, int V_full, int d, const int32_t* keep_ids, int V_trim,
                          void* W_trim, cudaStream_t st);

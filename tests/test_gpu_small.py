@@ -64,6 +64,23 @@ def test_coverage_bit_exact(vt, oracle, V, N, Vt, offset):
     assert (covered, frac) == oracle.coverage(tok[offset:], keep, V)
 
 
+def test_coverage_in_two_steps_matches_the_one_call_form(vt, oracle):
+    """vt_coverage_enqueue + vt_coverage_result: two enqueues back to back on different streams' worth of data,
+    each result read from its own workspace; a large stream so that every CTA runs the unrolled loop and its tail."""
+    V = 128256
+    rng = np.random.default_rng(12)
+    toks = [rng.integers(-2, V + 2, size=n).astype(np.int32) for n in (3_000_017, 70_001)]
+    keep = rng.permutation(V)[:13264].astype(np.int32)
+    keep_dev = dev_i32(keep)
+    devs = [dev_i32(t) for t in toks]
+    wss = [torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda") for _ in toks]
+    for t, ws in zip(devs, wss):
+        vt.vt_coverage_enqueue(t, keep_dev, V, ws)
+    assert vt.vt_last_launch_count() == 2
+    for t, ws in zip(toks, wss):
+        assert vt.vt_coverage_result(ws, t.size) == oracle.coverage(t, keep, V)
+
+
 def test_coverage_zipf_stream_and_validate(vt, oracle):
     V = inputs.V_LLAMA3
     tok = inputs.zipf_token_stream(V, 1.1, 574_168, seed=2)               # combined size of Table 4's streams
