@@ -126,8 +126,10 @@ vt_status vt_validate_keep_ids(const int32_t* keep_ids, int V_trim, int V_full,
  *   vt_draft_head_path with VT_HEAD_STATIC_WEIGHTS relaxes this for W_trim only: the caller declares that
  *   nothing earlier in the stream writes W_trim (it was written once, e.g. by vt_compact_head, and the
  *   stream or device was synchronised afterwards - the usual state of model weights in a serving loop).
- *   Weight tiles are then requested before the wait, which hides the first memory round trip behind the
- *   previous call's tail.  h, d2t, the workspace and the outputs keep full stream-order semantics.
+ *   A kernel may then request weight tiles before the wait, which hides the first memory round trip behind
+ *   the previous call's tail (the CUDA-core path for one or two draft rows does; the tensor-core paths
+ *   measured no gain and ignore the option).  h, d2t, the workspace and the outputs keep full stream-order
+ *   semantics.
  * Asynchronous: no host synchronisation.  A device-side wait that ran out is reported by
  * vt_last_status on the same workspace; after VT_ERR_TIMEOUT run vt_workspace_init again before
  * the workspace is reused (arrival counters may be left mid-count).

@@ -229,6 +229,122 @@ __device__ __forceinline__ void vals_insert(float (&g)[KR], float x) {
     g[0] = fmaxf(g[0], x);
 }
 
+
+// 16 consecutive logits of a draft row from shared memory (columns c .. c + 15, c a multiple of 4 floats from a
+// 16-byte aligned row); columns at or past `ce` come back as -inf.
+__device__ __forceinline__ void row_load16(const float* rowp, int c, int ce, float (&x)[16]) {
+#pragma unroll
+    for (int u4 = 0; u4 < 4; ++u4) {
+        const float4 f = *reinterpret_cast<const float4*>(rowp + c + 4 * u4);
+        x[4 * u4 + 0] = f.x; x[4 * u4 + 1] = f.y; x[4 * u4 + 2] = f.z; x[4 * u4 + 3] = f.w;
+    }
+    const int left = ce - c;
+    if (left < 16) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) x[e] = e < left ? x[e] : -INFINITY;
+    }
+}
+
+// Running log-sum-exp of one draft row over its columns [cb, ce) (at most 128): (max, sum of exp(x - max)).
+__device__ __forceinline__ void row_scan_lse(const float* rowp, int cb, int ce, float& mx, float& ssum) {
+    const int nch = (ce - cb + 15) >> 4;
+    for (int q = 0; q < nch; ++q) {
+        float x[16];
+        row_load16(rowp, cb + 16 * q, ce, x);
+        float cm = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+        cm = fmaxf(cm, fmaxf(fmaxf(fmaxf(x[8], x[9]), fmaxf(x[10], x[11])), fmaxf(fmaxf(x[12], x[13]), fmaxf(x[14], x[15]))));
+        const float nm = fmaxf(mx, cm);
+        const float nml = nm * kLog2e;
+        float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) {
+            a0 += ex2_approx(fmaf(x[e], kLog2e, -nml));             // exp(-inf) = 0
+            a1 += ex2_approx(fmaf(x[e + 1], kLog2e, -nml));
+        }
+        ssum = ssum * ex2_approx((mx - nm) * kLog2e) + (a0 + a1);   // first chunk: 0 * 0
+        mx = nm;
+    }
+}
+
+constexpr int kRowQueue = 64;      // candidate columns a thread can queue per scan; more than that and the warp inserts every column
+
+// Top-k update of one draft row by ONE thread over the row's columns [cb, ce) in shared memory (at most 128
+// columns; column c is vocabulary row idx0 + c).  `full` says whether the thread's list already holds KR entries
+// (the same in every lane of the warp: all lanes have scanned equally many logits).
+//   list full:      candidates are the logits above the list's last entry (strictly: a later row loses a tie);
+//   first scan of a long range: the KR-th largest of the maxima of groups of 4 or 8 logits has at least KR logits
+//                   at or above it, so nothing below it can be among the KR best: candidates are the logits not
+//                   below that bound;
+//   first scan of a short range: every logit goes through the list.
+// The candidates' columns are compacted into the thread's queue (`queue`: the thread's first byte, entries 128
+// bytes apart; branch-free: every column is stored and a candidate keeps its slot), then inserted one per turn
+// of a loop that runs for the busiest lane's count, each turn's column and logit fetched ahead of its
+// insertion.  The compare-and-select pipe runs at half rate, which makes the insertion (5 such operations
+// per list entry) the cost of this function: it is spent on the candidates only.  All lanes must call it.
+template <int KR>
+__device__ __forceinline__ void row_scan_topk(const float* rowp, int cb, int ce, int idx0, bool full, float (&v)[KR],
+                                              int (&ix)[KR], unsigned char* queue) {
+    const int n = ce - cb, nch = (n + 15) >> 4;
+    const int gs = full ? 0 : n >= 8 * (KR + 2) ? 8 : n >= 4 * (KR + 2) ? 4 : 0;
+    bool all = !full && gs == 0;
+    int cnt = 0;
+    if (!all) {
+        float tau = v[KR - 1];
+        if (!full) {       // bound from group maxima: at least KR + 2 whole groups exist
+            float g[KR];
+#pragma unroll
+            for (int j = 0; j < KR; ++j) g[j] = -INFINITY;
+            for (int q = 0; q < nch; ++q) {
+                float x[16];
+                row_load16(rowp, cb + 16 * q, ce, x);
+                if (gs == 8) {
+#pragma unroll
+                    for (int u8 = 0; u8 < 2; ++u8)
+                        vals_insert<KR>(g, fmaxf(fmaxf(fmaxf(x[8 * u8], x[8 * u8 + 1]), fmaxf(x[8 * u8 + 2], x[8 * u8 + 3])),
+                                                 fmaxf(fmaxf(x[8 * u8 + 4], x[8 * u8 + 5]), fmaxf(x[8 * u8 + 6], x[8 * u8 + 7]))));
+                } else {
+#pragma unroll
+                    for (int u4 = 0; u4 < 4; ++u4)
+                        vals_insert<KR>(g, fmaxf(fmaxf(x[4 * u4], x[4 * u4 + 1]), fmaxf(x[4 * u4 + 2], x[4 * u4 + 3])));
+                }
+            }
+            tau = g[KR - 1];
+        }
+        for (int q = 0; q < nch; ++q) {
+            float x[16];
+            row_load16(rowp, cb + 16 * q, ce, x);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                queue[min(cnt, kRowQueue - 1) * 128] = (unsigned char)(16 * q + e);
+                cnt += (full ? x[e] > tau : x[e] >= tau) ? 1 : 0;
+            }
+        }
+        const int most = (int)__reduce_max_sync(0xFFFFFFFFu, (unsigned)cnt);
+        all = most > kRowQueue;
+        if (!all) {
+            // turn i inserts the lane's i-th candidate; its column was fetched two turns earlier, its logit one
+            int c1 = queue[0], c2 = queue[128];
+            float x1 = rowp[cb + (cnt > 0 ? c1 : 0)];
+            for (int i = 0; i < most; ++i) {
+                const float xv = i < cnt ? x1 : -INFINITY;         // -inf beats nothing
+                const int xi = idx0 + cb + c1;
+                c1 = c2;
+                x1 = rowp[cb + (i + 1 < cnt ? c1 : 0)];
+                c2 = queue[min(i + 2, kRowQueue - 1) * 128];
+                rows_insert<KR>(v, ix, xv, xi);
+            }
+        }
+    }
+    if (all) {
+        for (int q = 0; q < nch; ++q) {
+            float x[16];
+            row_load16(rowp, cb + 16 * q, ce, x);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) rows_insert<KR>(v, ix, x[e], idx0 + cb + 16 * q + e);
+        }
+    }
+}
+
 // Register-list length for a top-k of k: the smallest instantiated length that holds k entries, 0 if none does.
 __host__ __device__ inline int topk_list_regs(int k) { return k <= 4 ? 4 : k <= 8 ? 8 : k <= 10 ? 10 : k <= 16 ? 16 : 0; }
 

@@ -43,7 +43,6 @@ struct RowsParams {
     HeadOut out;
     int m_begin, m_count;     // draft rows of this pass: m_count <= 128 * MT
     int MT;                   // A tiles of 128 draft rows: 1 or 2
-    int early_weights;        // 1: weight boxes may be requested before the dependency wait (W_trim declared constant)
     int d, nk;                // nk = 64-column k-blocks
     int NT;                   // vocabulary rows per tile: a multiple of 16, <= 256 (<= 128 with two A tiles)
     int kbw;                  // k-blocks one stage of the weight ring holds (one barrier hand-over per stage)
@@ -127,9 +126,8 @@ head_rows_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above touched only shared memory, tensor memory and kernel parameters.  Every thread now waits
-    // until the previous kernel in the stream has completed - except that the thread producing the weight ring,
-    // when the caller has declared W_trim constant, first fills that ring.
-    if (!(warp == w_warp && lane == 0)) grid_dependency_wait();
+    // until the previous kernel in the stream has completed.
+    grid_dependency_wait();
     if (tid == 0) grid_launch_dependents();
 
     auto fail = [&]() {
@@ -151,12 +149,9 @@ head_rows_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                     tma_load_2d_hint(base + ((uint32_t)s * (uint32_t)kbw + (uint32_t)kb) * p.b_slot, &tmW, (ks + kb) * kBoxK,
                                      row_begin + t * NT, bar, stream_once);
             };
-            const int pre = p.early_weights ? min(SW, total) : 0;
-            for (int q = 0; q < pre; ++q) issue(q, q);
-            grid_dependency_wait();
-            int s = pre == SW ? 0 : pre, issued = pre;
-            uint32_t wrap = pre == SW ? 1u : 0u;  // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
-            for (int q = pre; q < total; ++q) {
+            int s = 0, issued = 0;
+            uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
+            for (int q = 0; q < total; ++q) {
                 if (wrap > 0 && !mbar_wait(bar_wempty + 8u * s, (wrap - 1) & 1u)) { fail(); break; }
                 if (*abort_flag) break;
                 issue(q, s);
@@ -498,7 +493,6 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         const int mc = pass_rows(m0, &p);
         p.out = c.out;
         p.m_begin = m0;
-        p.early_weights = c.static_weights;
         CUtensorMap tmW, tmH;
         r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, p.NT);
         if (r != VT_OK) return r;

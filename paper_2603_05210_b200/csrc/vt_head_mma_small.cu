@@ -19,7 +19,7 @@
 //               would put several round trips to L2 per row on the critical path: the kernel then only writes
 //               the records and a one-warp-per-row merge kernel follows it.
 //   next warp   TMA producer: boxes of 64 columns x tile-height rows of W (and the k-block of h) into a
-//               shared-memory ring; it starts before the dependency wait (W_trim is a model constant)
+//               shared-memory ring
 //   last warp   MMA issuer: four K=16 tcgen05.mma (M=128, N) per 64-column k-block, tcgen05.commit frees the ring
 //               stage; two accumulator buffers in TMEM
 // Short tiles (a CTA with at most 64 rows: V_trim up to about 9,500) would waste the MMA: it costs the same 60-80
@@ -60,7 +60,6 @@ struct SmallParams {
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
     uint32_t tmem_cols;       // allocation: 2 accumulators of N columns, a power of two >= 32
     int d, nk;                // nk = 64-column k-blocks
-    int early_weights;        // 1: weight boxes may be requested before the dependency wait (W_trim declared constant)
     int G;                    // k-blocks folded into one MMA: 128 / (tile height rounded up to 32 or 64), or 1
     int NG;                   // accumulator columns per folded k-block = rows of an h block: 8 (M <= 8), else M rounded up to 16
     int nsb;                  // MMA steps along d: ceil(nk / G) "super-blocks" of G k-blocks
@@ -173,12 +172,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above touched only shared memory, tensor memory and kernel parameters, so under programmatic
-    // dependent launch it overlaps the previous kernel's tail.  Every thread but the producer now waits until the
-    // previous kernel has completed and its writes are visible; nothing of h, d2t, the workspace or the outputs is
-    // touched before that.  The producing thread waits inside its own branch: when the caller has declared W_trim
-    // a constant of the model it first fills the ring with weight boxes - while the previous call still merges -
-    // so that the ring is full when the first MMA may be issued.
-    if (!(warp == producer_warp && lane == 0)) grid_dependency_wait();
+    // dependent launch it overlaps the previous kernel's tail.  Every thread now waits until the previous kernel
+    // has completed and its writes are visible; no global memory is touched before that.  (Requesting weight tiles ahead of this wait, for weights the caller declares constant,
+    // was measured to cost 1-4 % here: the early requests compete with the previous call's last tiles.)
+    grid_dependency_wait();
     if (tid == 0) grid_launch_dependents();
 
     auto fail = [&]() {
@@ -194,39 +191,31 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             const int total = ntiles * spt;                 // ring stages of this CTA, in issue order
             const uint64_t stream_once = l2_policy_evict_first();
             const uint32_t h_tx = p.h_resident ? 0u : p.h_blk;
-            // stage q of the CTA's sequence into ring slot s: the weight boxes and/or the matching blocks of h
-            auto issue = [&](int q, int s, bool weights, bool hidden) {
+            // stage q of the CTA's sequence into ring slot s: the weight boxes and the matching blocks of h
+            auto issue = [&](int q, int s) {
                 const int t = q / spt, ks = (q - t * spt) * kbs;
                 const int row0 = row_begin + t * TH;
                 const int nb = min(kbs, nsb - ks);
                 const uint32_t bar = bar_full + 8u * s;
-                if (weights) mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + h_tx));
+                mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + h_tx));
                 for (int kb = 0; kb < nb; ++kb) {
                     const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
                     // k-block KF * (ks + kb) + g goes to lanes g * (128 / KF) ...; one past d is all zero fill
-                    if (weights)
-                        for (int g = 0; g < KF; ++g)
-                            tma_load_2d_hint(dst + (uint32_t)g * p.sub_bytes, &tmW, ((ks + kb) * KF + g) * kBoxK, row0, bar,
-                                             stream_once);
-                    if (hidden && !p.h_resident)      // the matching k-blocks of h, one block after the other behind the weights
+                    for (int g = 0; g < KF; ++g)
+                        tma_load_2d_hint(dst + (uint32_t)g * p.sub_bytes, &tmW, ((ks + kb) * KF + g) * kBoxK, row0, bar,
+                                         stream_once);
+                    if (!p.h_resident)                // the matching k-blocks of h, one block after the other behind the weights
                         for (int g = 0; g < KF; ++g)
                             tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK,
                                         p.m_begin, bar);
                 }
             };
-            // With weights the caller declared constant, the ring is filled with weight boxes ahead of the
-            // dependency wait - each stage's barrier already expects the bytes of its h blocks, which are only
-            // requested after the wait, like every other read of what the previous kernel may have written.
-            const int pre = p.early_weights ? min(S, total) : 0;
-            for (int q = 0; q < pre; ++q) issue(q, q, true, false);
-            grid_dependency_wait();
-            for (int q = 0; q < pre; ++q) issue(q, q, false, true);
-            int s = pre == S ? 0 : pre, issued = pre;
-            uint32_t wrap = pre == S ? 1u : 0u;  // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
-            for (int q = pre; q < total; ++q) {
+            int s = 0, issued = 0;
+            uint32_t wrap = 0;          // times the ring has wrapped: stage s is free once its (wrap-1)-th use retired
+            for (int q = 0; q < total; ++q) {
                 if (wrap > 0 && !mbar_wait(bar_empty + 8u * s, (wrap - 1) & 1u)) { fail(); break; }
                 if (*abort_flag) break;
-                issue(q, s, true, true);
+                issue(q, s);
                 ++issued;
                 if (++s == S) { s = 0; ++wrap; }
             }
@@ -379,120 +368,9 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             // previous tile again: whatever is computed from it belongs to a call that reports the time-out.
             const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
             const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
-            const int nch = (n + 15) >> 4;
-            auto load16 = [&](int q, float (&x)[16]) {             // chunk q of the range, columns past it as -inf
-                const int c = cb + 16 * q;
-#pragma unroll
-                for (int u4 = 0; u4 < 4; ++u4) {
-                    const float4 f = *reinterpret_cast<const float4*>(rowp + c + 4 * u4);
-                    x[4 * u4 + 0] = f.x; x[4 * u4 + 1] = f.y; x[4 * u4 + 2] = f.z; x[4 * u4 + 3] = f.w;
-                }
-                const int left = ce - c;
-                if (left < 16) {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) x[e] = e < left ? x[e] : -INFINITY;
-                }
-            };
-            if (works && n > 0 && !scanner) {
-                // running log-sum-exp of the row over these columns: (max, sum of exp(x - max))
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    if (q < nch) {
-                        float x[16];
-                        load16(q, x);
-                        float cm = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
-                        cm = fmaxf(cm, fmaxf(fmaxf(fmaxf(x[8], x[9]), fmaxf(x[10], x[11])), fmaxf(fmaxf(x[12], x[13]), fmaxf(x[14], x[15]))));
-                        const float nm = fmaxf(mx, cm);
-                        const float nml = nm * kLog2e;
-                        float a0 = 0.0f, a1 = 0.0f;
-#pragma unroll
-                        for (int e = 0; e < 16; e += 2) {
-                            a0 += ex2_approx(fmaf(x[e], kLog2e, -nml));             // exp(-inf) = 0
-                            a1 += ex2_approx(fmaf(x[e + 1], kLog2e, -nml));
-                        }
-                        ssum = ssum * ex2_approx((mx - nm) * kLog2e) + (a0 + a1);   // first chunk: 0 * 0
-                        mx = nm;
-                    }
-                }
-            }
-            if (works && n > 0 && scanner) {
-                const bool full = seen >= KL;
-                const int gs = full ? 0 : n >= 8 * (KL + 2) ? 8 : n >= 4 * (KL + 2) ? 4 : 0;
-                if (!full && gs == 0) {
-                    // a short first range: every logit goes through the list
-                    for (int q = 0; q < nch; ++q) {
-                        float x[16];
-                        load16(q, x);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) rows_insert<KL>(v, ix, x[e], row0 + cb + 16 * q + e);
-                    }
-                } else {
-                    float tau = v[KL - 1];
-                    if (!full) {       // bound from group maxima: at least KL + 2 whole groups exist
-                        float g[KL];
-#pragma unroll
-                        for (int j = 0; j < KL; ++j) g[j] = -INFINITY;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            if (q < nch) {
-                                float x[16];
-                                load16(q, x);
-                                if (gs == 8) {
-#pragma unroll
-                                    for (int u8 = 0; u8 < 2; ++u8)
-                                        vals_insert<KL>(g, fmaxf(fmaxf(fmaxf(x[8 * u8], x[8 * u8 + 1]), fmaxf(x[8 * u8 + 2], x[8 * u8 + 3])),
-                                                                 fmaxf(fmaxf(x[8 * u8 + 4], x[8 * u8 + 5]), fmaxf(x[8 * u8 + 6], x[8 * u8 + 7]))));
-                                } else {
-#pragma unroll
-                                    for (int u4 = 0; u4 < 4; ++u4)
-                                        vals_insert<KL>(g, fmaxf(fmaxf(x[4 * u4], x[4 * u4 + 1]), fmaxf(x[4 * u4 + 2], x[4 * u4 + 3])));
-                                }
-                            }
-                        }
-                        tau = g[KL - 1];
-                    }
-                    // candidates: above the list's last entry (a later row loses a tie), or not below the bound
-                    uint32_t mk[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (q < nch) {
-                            float x[16];
-                            load16(q, x);
-                            uint32_t bits = 0;
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) bits |= (full ? x[e] > tau : x[e] >= tau) ? (1u << e) : 0u;
-                            mk[q >> 1] |= bits << (16 * (q & 1));
-                        }
-                    }
-                    // one candidate per lane and turn; the next one's logit is fetched while this one is inserted
-                    auto next = [&](float& xv, int& xi) {
-                        xv = -INFINITY;
-                        xi = 0;
-                        const int w = mk[0] ? 0 : mk[1] ? 1 : mk[2] ? 2 : 3;
-                        const uint32_t word = w == 0 ? mk[0] : w == 1 ? mk[1] : w == 2 ? mk[2] : mk[3];
-                        if (word != 0u) {
-                            const int c = cb + 32 * w + __ffs(word) - 1;
-                            const uint32_t rest = word & (word - 1u);
-                            mk[0] = w == 0 ? rest : mk[0];
-                            mk[1] = w == 1 ? rest : mk[1];
-                            mk[2] = w == 2 ? rest : mk[2];
-                            mk[3] = w == 3 ? rest : mk[3];
-                            xv = rowp[c];
-                            xi = row0 + c;
-                        }
-                    };
-                    bool more = __any_sync(0xFFFFFFFFu, (mk[0] | mk[1] | mk[2] | mk[3]) != 0u);
-                    float nxv;
-                    int nxi;
-                    next(nxv, nxi);
-                    while (more) {
-                        const float xv = nxv;
-                        const int xi = nxi;
-                        more = __any_sync(0xFFFFFFFFu, (mk[0] | mk[1] | mk[2] | mk[3]) != 0u);
-                        next(nxv, nxi);
-                        rows_insert<KL>(v, ix, xv, xi);            // -inf beats nothing
-                    }
-                }
+            if (works && n > 0) {
+                if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + tid);
+                else row_scan_lse(rowp, cb, ce, mx, ssum);
             }
             seen += max(n, 0);
             epi_barrier(256);                                      // the buffer may be overwritten
@@ -708,7 +586,8 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, in
     p->n_epi = KR > 0 ? 8 : M > 8 ? kSmMaxEpiWarps : 8;
     p->merge_in_kernel = KR == 0 && M <= p->n_epi;
     p->scratch_stride = (uint32_t)(kSmCand - VT_MAX_K + k) * 8u;
-    const size_t scratch_bytes = KR > 0 ? 0 : ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
+    // thread-per-row: the scanners' candidate queues, kRowQueue entries of one byte for each of 128 threads
+    const size_t scratch_bytes = KR > 0 ? (size_t)kRowQueue * 128 : ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
     const size_t bar_bytes = (size_t)(2 * kSmMaxStages + 4 + kHParts + 1) * 8 + 16;
     const size_t common = 1024 + lg_bytes + list_bytes + scratch_bytes + bar_bytes + 128;
     // h resident only for M <= 8 (8 rows per k-block) and short tiles, where little is streamed and the fold by two
@@ -798,7 +677,6 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
         small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p, &KR);
         p.out = c.out;
         p.m_begin = m0;
-        p.early_weights = c.static_weights;
         if (c.M > kSmMaxM) p.merge_in_kernel = 0;       // row tickets serve single-pass calls only
         merge_after = !p.merge_in_kernel;
         CUtensorMap tmW, tmH;
