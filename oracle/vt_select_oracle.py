@@ -9,6 +9,7 @@ Plain numpy in fp64 / int64, one function per definition of the paper's Method s
   utility         U(k) = alpha C(k) + (1 - alpha) R(k)                                         Eq. 4
   penalised       U~(k) = U(k) if C(k) >= c_min else -1                                        Eq. 5
   selection       k* = argmax_{k in [k_min, k_max]} U~(k), the smallest k among equal maxima   Eq. 1
+  unique coverage fraction of the DISTINCT ids of the stream that the top-k keeps               Table 4 caption
 
 The paper searches k with 100 TPE trials; an exhaustive scan over every k gives the exact optimum of the
 same objective and is what both this oracle and the CUDA path compute.  It shares no code with the CUDA path.
@@ -44,6 +45,14 @@ def coverage_curve(f: np.ndarray, order: np.ndarray) -> np.ndarray:
     return cum.astype(np.float64) / np.float64(cum[-1])
 
 
+def unique_coverage_curve(f: np.ndarray, order: np.ndarray) -> np.ndarray:
+    """Unique coverage for k = 1..V (index k-1): of the distinct ids that occur in the stream (f > 0), the
+    fraction that lies in the top-k.  Table 4 reports it beside the frequency-weighted coverage of Eq. 2."""
+    occurs = (f[order] > 0).astype(np.int64)
+    distinct = int(occurs.sum())
+    return np.cumsum(occurs).astype(np.float64) / np.float64(distinct)
+
+
 def fixed_flops(d: int, attention: float, feed_forward: float) -> float:
     """F_fixed: feature fusion (3d -> d projection, 2 * 3d * d FLOPs) + attention + feed-forward (Table 1 gives the last two)."""
     return 2.0 * (3 * d) * d + attention + feed_forward
@@ -75,4 +84,5 @@ def select(token_ids: np.ndarray, V: int, d: int, F_fixed: float, alpha: float, 
     window = Ut[lo - 1:hi]
     k_star = lo + int(np.argmax(window))          # argmax returns the first (smallest k) of equal maxima
     return {"f": f, "order": order, "sorted_counts": f[order], "C": C, "R": R, "U": U, "U_pen": Ut, "k_star": k_star,
-            "C_star": float(C[k_star - 1]), "R_star": float(R[k_star - 1]), "U_star": float(Ut[k_star - 1])}
+            "C_star": float(C[k_star - 1]), "R_star": float(R[k_star - 1]), "U_star": float(Ut[k_star - 1]),
+            "unique_star": float(unique_coverage_curve(f, order)[k_star - 1])}
