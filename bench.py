@@ -424,7 +424,8 @@ def once_per_model(vt, torch, W_full, keep, W_trim, tok_dev, tokens, d, V, peak_
         sel = vt.vt_select_vocab(tok_dev, V, d, F_fixed, 0.5, 0.9, 1000, 64000, workspace=sel_ws)
     out["select_vocab_us_incl_sync"] = round((time.perf_counter() - t0) * 2e5, 1)
     out["select_vocab"] = {"alpha": 0.5, "c_min": 0.9, "k_range": [1000, 64000], "k_star": sel["k_star"],
-                           "C": round(sel["C"], 6), "R": round(sel["R"], 6), "U": round(sel["U"], 6)}
+                           "C": round(sel["C"], 6), "R": round(sel["R"], 6), "U": round(sel["U"], 6),
+                           "unique_coverage": round(sel["unique"], 6)}
     return out
 
 

@@ -171,6 +171,24 @@ vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32
 vt_status vt_last_status(void* workspace, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Feature fusion of an EAGLE-style draft (Section 2.3, component 1: the layer that projects the concatenated
+ * hidden states of several target-model layers into the hidden dimension; Table 1, first row, 2 * 3d * d
+ * FLOPs - part of the fixed cost F_fixed of Eq. 3, independent of the vocabulary):
+ *
+ *   fused[m, i] = bf16( sum_j h3[m, j] * W_fuse[i, j] )     fp32 accumulation of exact bf16 products, rounded
+ *                                                           once, to nearest-even
+ *
+ *   h3      dev [M, d_in]  bf16, 16-byte aligned (d_in = 3d for three concatenated layers)
+ *   W_fuse  dev [d_out, d_in] bf16, 16-byte aligned, row-major (one row per output feature)
+ *   fused   dev [M, d_out] bf16 (out)
+ *   workspace  a draft-head workspace of at least vt_workspace_bytes(M, 1) bytes (only its status word is used)
+ * d_in % 8 == 0, d_in >= 8.  It runs the head's contraction kernels with an epilogue that only stores, so the
+ * fixed part of a draft step can be timed on the same footing as the vocabulary-dependent part.
+ * Asynchronous; stream order as for vt_draft_head. */
+vt_status vt_fuse_features(const void* h3, const void* W_fuse, int M, int d_in, int d_out,
+                           void* fused, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Coverage of a token stream by the kept set (Eq. 2 with f(v) = occurrences of v in the
  * stream; the "frequency coverage" of Table 4):
  *
@@ -216,6 +234,8 @@ vt_status vt_coverage_result(void* workspace, int64_t N,
  *                                       vocabulary, i.e. keep_ids / d2t for the calls above
  *   cum_counts dev [V_full] uint64 (out) or NULL: cum_counts[k-1] = occurrences covered by the top k
  *   k_star     host (out);  C_star, R_star, U_star  host (out), each may be NULL
+ *   unique_star host (out) or NULL: of the distinct ids that occur in the stream, the fraction that the top k*
+ *              keeps (the "unique coverage" Table 4 reports beside Eq. 2's frequency-weighted coverage)
  *   workspace  dev, 256-byte aligned, vt_select_workspace_bytes(V_full); contents are overwritten
  * 1 <= k_min <= k_max <= V_full, 0 <= alpha <= 1, F_fixed >= 0, d >= 1, N < 2^32 (frequencies are counted in
  * 32 bits; a longer stream gives VT_ERR_SHAPE).  SYNCHRONISES the stream.
@@ -224,7 +244,7 @@ size_t    vt_select_workspace_bytes(int V_full);
 vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed,
                           double alpha, double c_min, int k_min, int k_max,
                           int32_t* ranked_ids, uint64_t* cum_counts,
-                          int* k_star, double* C_star, double* R_star, double* U_star,
+                          int* k_star, double* C_star, double* R_star, double* U_star, double* unique_star,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /* vt_coverage for callers that must not allocate device memory.  (The paper has no counterpart: this

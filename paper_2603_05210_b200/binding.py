@@ -42,9 +42,10 @@ SYMBOLS = {
     "vt_coverage_result": (_i, [_p, _i64, _p, _p, _p]),
     "vt_select_workspace_bytes": (_sz, [_i]),
     "vt_select_vocab": (_i, [_p, _i64, _i, _i, ctypes.c_double, ctypes.c_double, ctypes.c_double, _i, _i, _p, _p, _p, _p, _p,
-                            _p, _p, _sz, _p]),
+                            _p, _p, _p, _sz, _p]),
     "vt_coverage_static": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p]),
     "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
+    "vt_fuse_features": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p]),
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
     "vt_vocab_maps": (_i, [_p, _i, _i, _p, _p, _p]),
     "vt_last_launch_count": (_i, []),
@@ -243,12 +244,13 @@ def vt_select_vocab(token_ids: torch.Tensor, V_full: int, d: int, F_fixed: float
     if workspace is None:
         workspace = torch.empty(vt_select_workspace_bytes(V_full), dtype=torch.uint8, device=dev)
     k_star = ctypes.c_int(0)
-    C, R, U = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_double(0)
+    C, R, U, uq = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_double(0), ctypes.c_double(0)
     _check(lib().vt_select_vocab(token_ids.data_ptr() if token_ids.numel() else None, token_ids.numel(), V_full, d,
                                  float(F_fixed), float(alpha), float(c_min), k_min, k_max, ranked.data_ptr(), _ptr(cum),
                                  ctypes.addressof(k_star), ctypes.addressof(C), ctypes.addressof(R), ctypes.addressof(U),
-                                 workspace.data_ptr(), workspace.numel(), _stream()), "vt_select_vocab")
-    out = {"k_star": int(k_star.value), "C": float(C.value), "R": float(R.value), "U": float(U.value), "ranked_ids": ranked}
+                                 ctypes.addressof(uq), workspace.data_ptr(), workspace.numel(), _stream()), "vt_select_vocab")
+    out = {"k_star": int(k_star.value), "C": float(C.value), "R": float(R.value), "U": float(U.value),
+           "unique": float(uq.value), "ranked_ids": ranked}
     if want_cum:
         out["cum_counts"] = cum
     return out
@@ -278,6 +280,24 @@ def vt_debug_logits(h: torch.Tensor, W_trim: torch.Tensor, path: int = VT_PATH_A
     _check(lib().vt_debug_logits(h.data_ptr(), W_trim.data_ptr(), M, d, Vt, logits.data_ptr(), ws.data_ptr(),
                                  ws.numel(), _stream(), path), "vt_debug_logits")
     return logits
+
+
+def vt_fuse_features(h3: torch.Tensor, W_fuse: torch.Tensor, *, out: torch.Tensor | None = None,
+                     workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """fused [M, d_out] bf16 = h3 [M, d_in] x W_fuse[d_out, d_in]^T, fp32 accumulation, one rounding to bf16."""
+    h3 = _bf16(h3, "h3")
+    W_fuse = _bf16(W_fuse, "W_fuse")
+    M, d_in = h3.shape
+    d_out, d2 = W_fuse.shape
+    if d2 != d_in:
+        raise ValueError("h3 and W_fuse disagree on d_in")
+    if out is None:
+        out = torch.empty((M, d_out), dtype=h3.dtype, device=h3.device)
+    if workspace is None:
+        workspace = new_workspace(vt_workspace_bytes(M, 1), h3.device)
+    _check(lib().vt_fuse_features(h3.data_ptr(), W_fuse.data_ptr(), M, d_in, d_out, out.data_ptr(), workspace.data_ptr(),
+                                  workspace.numel(), _stream()), "vt_fuse_features")
+    return out
 
 
 def vt_remap(draft_ids: torch.Tensor, d2t: torch.Tensor) -> torch.Tensor:

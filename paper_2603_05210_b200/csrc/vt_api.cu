@@ -126,7 +126,7 @@ static vt_status run_head(const HeadCall& c, cudaStream_t st, int path) {
         }
     }
     if (r != VT_OK) return r;
-    if (!merged) r = launch_merge_rowmajor(c.out, grid, st);
+    if (!merged && !c.out.store_only) r = launch_merge_rowmajor(c.out, grid, st);
     return r;
 }
 
@@ -350,6 +350,22 @@ vt_status vt_debug_logits(const void* h, const void* W_trim, int M, int d, int V
     HeadOut o = make_out(nullptr, M, V_trim, 1, tid, lp, nullptr, nullptr, logits, workspace);
     HeadCall c{h, W_trim, d, M, V_trim, o, 0};
     return run_head(c, (cudaStream_t)stream, path & VT_PATH_MASK);
+}
+
+vt_status vt_fuse_features(const void* h3, const void* W_fuse, int M, int d_in, int d_out, void* fused, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    g_launches = 0;
+    if (!h3 || !W_fuse || !fused) return VT_ERR_NULL;
+    if (d_in < 8 || d_in % 8 != 0 || d_out < 1 || M < 1) return VT_ERR_SHAPE;
+    if (!aligned(h3, 16) || !aligned(W_fuse, 16) || !aligned(fused, 2)) return VT_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < ws_total_bytes(M, 1)) return VT_ERR_WORKSPACE;
+    // the same contraction kernels as the head, rows of W_fuse in the place of vocabulary rows, with an epilogue
+    // that stores the rounded sums and nothing else
+    HeadOut o = make_out(nullptr, M, d_out, 1, nullptr, nullptr, nullptr, nullptr, nullptr, workspace);
+    o.rounded = reinterpret_cast<uint16_t*>(fused);
+    o.store_only = 1;
+    HeadCall c{h3, W_fuse, d_in, M, d_out, o, 0};
+    return run_head(c, (cudaStream_t)stream, VT_PATH_AUTO);
 }
 
 vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim, int32_t* target_ids,

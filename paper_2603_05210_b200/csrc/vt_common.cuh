@@ -3,6 +3,7 @@
 // top-k updates and the cross-CTA merge that ends a draft-head call.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -50,6 +51,8 @@ struct HeadOut {
     int32_t* draft_ids;   // may be null
     float* lse;           // may be null
     float* logits;        // debug: [M, Vt] fp32, null on the fast path
+    uint16_t* rounded;    // the contraction rounded to bf16, [M, Vt], null for the head
+    int store_only;       // 1: the contraction is the result (a plain projection): no top-k, no log-sum-exp, no records
     WsHeader* hdr;
     unsigned long long* recs;
     int M, k, Vt;
@@ -129,6 +132,15 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Writes x[m, col] where the caller asked for the contraction itself: fp32 for inspection, and / or rounded once
+// to bf16 (round-to-nearest-even) for a projection whose output feeds the next layer.
+__device__ __forceinline__ bool wants_logits(const HeadOut& o) { return o.logits != nullptr || o.rounded != nullptr; }
+__device__ __forceinline__ void store_logit(const HeadOut& o, int m, int col, float x) {
+    const size_t at = (size_t)m * o.Vt + col;
+    if (o.logits) o.logits[at] = x;
+    if (o.rounded) o.rounded[at] = __bfloat16_as_ushort(__float2bfloat16_rn(x));
 }
 
 // ------------------------------------------------------------------------------------------

@@ -207,13 +207,15 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
                 if (live && g0 + my_r < rows) {
                     const float x = v[0];
                     const int row = row_begin + t * SR + g0 + my_r;
-                    lse_update(mx, ssum, x);
-                    if (x > thr_x || filled < k) {     // rows reach this lane in ascending order: ties lose
-                        const unsigned long long kth = list_insert(my_list, 1, k, make_key(x, row));
-                        if (filled < k) ++filled;
-                        if (filled == k) thr_x = key_logit(kth);
+                    if (!p.out.store_only) {
+                        lse_update(mx, ssum, x);
+                        if (x > thr_x || filled < k) {     // rows reach this lane in ascending order: ties lose
+                            const unsigned long long kth = list_insert(my_list, 1, k, make_key(x, row));
+                            if (filled < k) ++filled;
+                            if (filled == k) thr_x = key_logit(kth);
+                        }
                     }
-                    if (p.out.logits) p.out.logits[(size_t)(p.m_begin + my_m) * Vt + row] = x;
+                    if (wants_logits(p.out)) store_logit(p.out, p.m_begin + my_m, row, x);
                 }
             }
             __syncwarp();
@@ -224,7 +226,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
     __syncthreads();
 
     // ---------------------------------------------------------------------- fold the CTA's lists: one warp per draft row
-    if (warp < p.m_count) {
+    if (warp < p.m_count && !p.out.store_only) {
         // lists of draft row `warp`: index (cw * NV + r * MP + warp), i.e. P1 = consumers * R lists, KS apart * MP
         const int m = warp;
         const int P1 = kGemvConsumers * R;

@@ -280,12 +280,12 @@ head_rows_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                     for (int c = 0; c < kRowsChunk; ++c)
                         if (c >= nv) x[c] = -INFINITY;
                 }
-                if (p.out.logits && live) {
-                    float* dst = p.out.logits + (size_t)row * Vt + row0 + c0;
+                if (wants_logits(p.out) && live) {
 #pragma unroll
                     for (int c = 0; c < kRowsChunk; ++c)
-                        if (c < nv) dst[c] = x[c];
+                        if (c < nv) store_logit(p.out, row, row0 + c0 + c, x[c]);
                 }
+                if (p.out.store_only) continue;
                 // running log-sum-exp of the row: (max, sum of exp(x - max))
                 float cm = x[0];
 #pragma unroll
@@ -339,7 +339,7 @@ head_rows_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
             if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
         }
         // the row's record: best k keys and (max, sum-exp); an unfilled entry is key 0
-        if (live) {
+        if (live && !p.out.store_only) {
             if (KR > 0) {
 #pragma unroll
                 for (int j = 0; j < KL; ++j)
@@ -508,7 +508,7 @@ vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid_out) {
         if (r != VT_OK) return r;
         m0 += mc;
     }
-    return launch_merge_rowmajor(c.out, grid, st);
+    return c.out.store_only ? VT_OK : launch_merge_rowmajor(c.out, grid, st);
 }
 
 }  // namespace vt

@@ -337,7 +337,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         float sum = 0.0f;
                         for (int gg = 0; gg < KF; ++gg) sum += partial[(gg * p.NG + m) * 64 + rr];
                         lg[m * kLgPitch + rr] = sum;
-                        if (p.out.logits) p.out.logits[(size_t)(p.m_begin + m) * Vt + row0 + rr] = sum;
+                        if (wants_logits(p.out)) store_logit(p.out, p.m_begin + m, row0 + rr, sum);
                     }
                 } else if (got) {
                     const int i = warp * 32 + lane;                // TMEM lane = vocabulary row of the tile
@@ -350,11 +350,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 #pragma unroll
                             for (int m = 0; m < 16; ++m)
                                 if (c1 + m < M) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(u[m]);
-                            if (p.out.logits) {
+                            if (wants_logits(p.out)) {
 #pragma unroll
                                 for (int m = 0; m < 16; ++m)
-                                    if (c1 + m < M)
-                                        p.out.logits[(size_t)(p.m_begin + c1 + m) * Vt + row0 + i] = __uint_as_float(u[m]);
+                                    if (c1 + m < M) store_logit(p.out, p.m_begin + c1 + m, row0 + i, __uint_as_float(u[m]));
                             }
                         }
                     }
@@ -368,7 +367,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             // previous tile again: whatever is computed from it belongs to a call that reports the time-out.
             const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
             const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
-            if (works && n > 0) {
+            if (works && n > 0 && !p.out.store_only) {
                 if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + tid);
                 else row_scan_lse(rowp, cb, ce, mx, ssum);
             }
@@ -388,7 +387,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             }
         }
         epi_barrier(256);
-        if (scanner && part == 0 && m_own < M) {
+        if (scanner && part == 0 && m_own < M && !p.out.store_only) {
             const int row = p.m_begin + m_own;                                 // among the call's draft rows
             // Q sorted lists: the best remaining key is the largest head, k times
             int pos[4] = {0, 0, 0, 0};
@@ -478,7 +477,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         float sum = 0.0f;
                         for (int gg = 0; gg < KF; ++gg) sum += part[(gg * p.NG + m) * 64 + rr];
                         lg[m * kLgPitch + rr] = sum;
-                        if (p.out.logits) p.out.logits[(size_t)(p.m_begin + m) * Vt + row0 + rr] = sum;
+                        if (wants_logits(p.out)) store_logit(p.out, p.m_begin + m, row0 + rr, sum);
                     }
                 }
                 got_tile = got;
@@ -499,11 +498,10 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 #pragma unroll
                             for (int m = 0; m < 16; ++m)
                                 if (c1 + m < mc) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(r[m]);
-                            if (p.out.logits) {
+                            if (wants_logits(p.out)) {
 #pragma unroll
                                 for (int m = 0; m < 16; ++m)
-                                    if (c1 + m < mc)
-                                        p.out.logits[(size_t)(p.m_begin + c0 + c1 + m) * Vt + row0 + i] = __uint_as_float(r[m]);
+                                    if (c1 + m < mc) store_logit(p.out, p.m_begin + c0 + c1 + m, row0 + i, __uint_as_float(r[m]));
                             }
                         }
                     }
@@ -514,7 +512,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     }
                 }
                 epi_barrier(n_epi * 32);                               // the chunk's logits are in shared memory
-                for (int m = c0 + warp; m < c0 + mc; m += n_epi) {
+                for (int m = c0 + warp; m < c0 + mc && !p.out.store_only; m += n_epi) {
                     const float tau = warp_topk_update<4>(lg + (m - c0) * kLgPitch, nv, row0, lists + (size_t)m * k, k,
                                                           tau_s[m], cbuf, ms_s + m, lane);
                     __syncwarp();
@@ -527,7 +525,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         // ------------------------------------------------------------------ publish, and merge if last
         // The warp owns its rows from the first tile to the outputs: record -> fence -> ticket; the warp that
         // draws the last ticket of a row (over all CTAs) merges that row.  No CTA-wide step in between.
-        for (int m = warp; m < M; m += n_epi) {
+        for (int m = warp; m < M && !p.out.store_only; m += n_epi) {
             const int row = p.m_begin + m;                             // among the call's draft rows
             const unsigned long long* list = lists + (size_t)m * k;
             for (int j = lane; j < k; j += 32) VT_ROW_KEYS(p.out, row, j)[cta] = list[j];
@@ -693,7 +691,7 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
         }
         if (r != VT_OK) return r;
     }
-    return merge_after ? launch_merge_rowmajor(c.out, grid, st) : VT_OK;
+    return merge_after && !c.out.store_only ? launch_merge_rowmajor(c.out, grid, st) : VT_OK;
 }
 
 }  // namespace vt

@@ -22,7 +22,8 @@ struct SelectResult {
     int pad;
     double C, R, U;
     unsigned long long total;
-    unsigned long long pad2[27];
+    double unique;              // of the distinct ids that occur, the fraction inside the top k*
+    unsigned long long pad2[26];
 };
 static_assert(sizeof(SelectResult) == 256, "one line");
 
@@ -137,15 +138,18 @@ __global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* _
                                                            SelectResult* result) {
     __shared__ unsigned long long warp_tot[32];
     __shared__ unsigned long long carry_s;
+    __shared__ unsigned int distinct_s;      // ids that occur at all (count > 0): they sort first
     __shared__ double best_u[32];
     __shared__ int best_k[32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) carry_s = 0ull;
+    if (tid == 0) { carry_s = 0ull; distinct_s = 0u; }
     __syncthreads();
     for (int c0 = 0; c0 < V; c0 += 1024) {              // inclusive prefix sum of the sorted counts
         const int i = c0 + tid;
         unsigned long long v = i < V ? (unsigned long long)(key_max - key_sorted[i]) : 0ull;
         if (i < V) ranked_ids[i] = val_sorted[i];
+        const unsigned int occurs = __ballot_sync(0xFFFFFFFFu, v > 0ull);
+        if (lane == 0 && occurs) atomicAdd(&distinct_s, (unsigned int)__popc(occurs));
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const unsigned long long n = __shfl_up_sync(0xFFFFFFFFu, v, o);
@@ -200,6 +204,10 @@ __global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* _
         result->R = br;
         result->U = bu;
         result->total = total;
+        // counts descend, so the ids that occur are exactly the first distinct_s of the ranking (Table 4's
+        // "unique coverage": kept distinct ids over all distinct ids)
+        const unsigned int distinct = distinct_s;
+        result->unique = distinct > 0 ? __ddiv_rn((double)min((unsigned int)max(bk, 0), distinct), (double)distinct) : 0.0;
     }
 }
 
@@ -217,8 +225,8 @@ extern "C" size_t vt_select_workspace_bytes(int V_full) {
 
 extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed, double alpha,
                                      double c_min, int k_min, int k_max, int32_t* ranked_ids, uint64_t* cum_counts,
-                                     int* k_star, double* C_star, double* R_star, double* U_star, void* workspace,
-                                     size_t workspace_bytes, void* stream) {
+                                     int* k_star, double* C_star, double* R_star, double* U_star, double* unique_star,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
     reset_launch_count();
     if (!ranked_ids || !k_star || (!token_ids && N > 0)) return VT_ERR_NULL;
     if (N > 0xFFFFFFFFll) return VT_ERR_SHAPE;                 // the histogram counts in 32 bits
@@ -272,5 +280,6 @@ extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_
     if (C_star) *C_star = host.C;
     if (R_star) *R_star = host.R;
     if (U_star) *U_star = host.U;
+    if (unique_star) *unique_star = host.unique;
     return VT_OK;
 }

@@ -93,9 +93,9 @@ def test_other_entry_points_reject_bad_arguments(vt):
     assert L.vt_remap(FAKE, FAKE, -1, 10, FAKE, None) == vt.VT_ERR_SHAPE
     assert L.vt_debug_logits(FAKE, FAKE, 1, 64, 10, None, FAKE, 1 << 20, None, 0) == vt.VT_ERR_NULL
     assert L.vt_workspace_init(None, 1024, None) == vt.VT_ERR_WORKSPACE
-    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 1, 100, None, None, FAKE, None, None, None, FAKE, 1 << 24, None) == vt.VT_ERR_NULL
-    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 0, 100, FAKE, None, FAKE, None, None, None, FAKE, 1 << 24, None) == vt.VT_ERR_SHAPE
-    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 1, 100, FAKE, None, FAKE, None, None, None, FAKE, 64, None) == vt.VT_ERR_WORKSPACE
+    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 1, 100, None, None, FAKE, None, None, None, None, FAKE, 1 << 24, None) == vt.VT_ERR_NULL
+    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 0, 100, FAKE, None, FAKE, None, None, None, None, FAKE, 1 << 24, None) == vt.VT_ERR_SHAPE
+    assert L.vt_select_vocab(FAKE, 10, 100, 64, 1e4, 0.5, 0.9, 1, 100, FAKE, None, FAKE, None, None, None, None, FAKE, 64, None) == vt.VT_ERR_WORKSPACE
     assert vt.vt_select_workspace_bytes(128256) >= 128256 * 28 and vt.vt_select_workspace_bytes(0) == 0
     assert L.vt_last_status(None, None) == vt.VT_ERR_WORKSPACE
     assert L.vt_draft_head_host(None, FAKE, FAKE, 1, 64, 10, 1, FAKE, FAKE, FAKE, 1 << 20, None) == vt.VT_ERR_NULL

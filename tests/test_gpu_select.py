@@ -26,6 +26,7 @@ def check(vt, tokens, V, d, F, alpha, c_min, k_min, k_max):
     assert np.array_equal(got["cum_counts"].cpu().numpy(), np.cumsum(ref["sorted_counts"]))
     assert got["k_star"] == ref["k_star"]
     assert got["C"] == ref["C_star"] and got["R"] == ref["R_star"] and got["U"] == ref["U_star"]
+    assert got["unique"] == ref["unique_star"]          # Table 4's unique coverage at k*: a ratio of two integers
     return got, ref
 
 

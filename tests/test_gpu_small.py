@@ -114,15 +114,37 @@ def test_remap_bit_exact(vt, oracle):
 
 
 def test_vocab_maps_bit_exact(vt):
+    """The draft-to-target offsets and the target-to-draft mask (Section 1) against the index-buffer oracle."""
+    from oracle import vt_maps_oracle as mo
     rng = np.random.default_rng(4)
     V, Vt = 128256, 13264
     keep = rng.permutation(V)[:Vt].astype(np.int32)
     off, mask = vt.vt_vocab_maps(dev_i32(keep), V)
-    assert np.array_equal(off.cpu().numpy(), keep - np.arange(Vt, dtype=np.int32))      # target = draft index + offset
-    want = np.zeros(V, dtype=np.uint8)
-    want[keep] = 1
-    assert np.array_equal(mask.cpu().numpy(), want)
+    assert np.array_equal(off.cpu().numpy(), mo.d2t_offsets(keep))
+    assert np.array_equal(mask.cpu().numpy(), mo.t2d_mask(keep, V))
     assert int(mask.sum()) == Vt
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M", [1, 8, 40])
+def test_head_with_offset_form_d2t(vt, oracle, path, M):
+    """VT_HEAD_D2T_OFFSETS: the head takes the offsets vt_vocab_maps wrote (target id = draft index + offset, the
+    form an EAGLE-3 style checkpoint stores) and must return the ids the oracle's offset remap gives."""
+    from oracle import vt_maps_oracle as mo
+    d, Vt, k, V = 512, 3001, 8, 50_000
+    h, W, _ = rand_case(M, d, Vt, seed=77 + M)
+    keep = np.sort(np.random.default_rng(M).permutation(V)[:Vt]).astype(np.int32)
+    off_dev, _ = vt.vt_vocab_maps(dev_i32(keep), V)
+    tid = torch.empty((M, k), dtype=torch.int32, device="cuda")
+    did = torch.empty((M, k), dtype=torch.int32, device="cuda")
+    ws = vt.new_workspace(vt.vt_workspace_bytes(M, k))
+    _, lp = vt.vt_draft_head(dev_bf16(h), dev_bf16(W), off_dev, k, workspace=ws, path=path, target_ids=tid, draft_ids=did,
+                             d2t_offsets=True)
+    assert vt.vt_last_status(ws) == vt.VT_OK
+    ora = oracle.draft_head(h, W, keep, k, want_logits=True)
+    got = {"target_ids": tid.cpu().numpy(), "logprobs": lp.cpu().numpy(), "draft_ids": did.cpu().numpy()}
+    assert np.array_equal(got["target_ids"], mo.remap_offsets(got["draft_ids"], mo.d2t_offsets(keep)))
+    parity.check_head(got, ora, keep, k)
 
 
 # ------------------------------------------------------------------------------ logits
