@@ -200,6 +200,12 @@ def time_head(vt, torch, h, W_copies, d2t, k, steps, warmup, path=0, use_graph=T
     return (out[0] if reps == 1 else out), launches
 
 
+def hold_gpu(torch, ms=8.0):
+    """Keeps the stream busy for a few milliseconds so that the host can enqueue what follows without the GPU ever
+    waiting for it: what is timed afterwards is device time, not the host's launch overhead."""
+    torch.cuda._sleep(int(ms * 1e-3 * 1.9e9))
+
+
 def time_isolated(vt, torch, h, W_copies, d2t, k, n_calls=ISOLATED_CALLS, path=0):
     """us of ONE call that follows an unrelated, ordinary kernel (an elementwise update of a 32 MB tensor: no
     programmatic early trigger, and it displaces part of L2), timed with a CUDA event pair per call on a cold
@@ -215,6 +221,7 @@ def time_isolated(vt, torch, h, W_copies, d2t, k, n_calls=ISOLATED_CALLS, path=0
         vt.vt_draft_head(h, W_copies[i % n], d2t, k, workspace=ws, path=path, target_ids=tid, logprobs=lp)
     pairs = []
     torch.cuda.synchronize()
+    hold_gpu(torch)          # the host enqueues all samples while the GPU is held, so no sample waits for the host
     for i in range(n_calls):
         filler.add_(1.0)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -306,13 +313,20 @@ def run_ours(args):
     h_host = torch.from_numpy(case.h.view(np.int16).copy()).pin_memory()
     tid_h = torch.empty((M, k), dtype=torch.int32).pin_memory()
     lp_h = torch.empty((M, k), dtype=torch.float32).pin_memory()
+    # the C entry point itself, with the pointers resolved once (what a C or C++ caller does every step)
+    c_call = vt.lib().vt_draft_head_host
+    w_ptrs = [w_.data_ptr() for w_ in copies]
+    fixed_args = (d2t.data_ptr(), M, d, Vt, k, tid_h.data_ptr(), lp_h.data_ptr(), hws.data_ptr(), hws.numel(),
+                  torch.cuda.current_stream().cuda_stream)
     for i in range(min(args.warmup, 50)):
-        vt.vt_draft_head_host(h_host, copies[i % nc], d2t, k, tid_h, lp_h, hws)
+        assert c_call(h_host.data_ptr(), w_ptrs[i % nc], *fixed_args) == vt.VT_OK
     torch.cuda.synchronize()
+    h_ptr = h_host.data_ptr()
     t0 = time.perf_counter()
     for i in range(e2e_steps):
-        vt.vt_draft_head_host(h_host, copies[i % nc], d2t, k, tid_h, lp_h, hws)
+        c_call(h_ptr, w_ptrs[i % nc], *fixed_args)
     e2e_us = (time.perf_counter() - t0) * 1e6 / e2e_steps
+    assert vt.vt_last_status(hws) == vt.VT_OK
     e2e_us = max_over_ranks(e2e_us, dist, "cuda")
 
     line = {
@@ -352,12 +366,55 @@ def run_ours(args):
             line["curve"] = latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, not args.no_graph)
             del W_full
             torch.cuda.empty_cache()
+            line["fixed_vs_head"] = fixed_vs_head(vt, torch, line["curve"], d, V, l2, peak_gbs)
             line["other_workloads"] = config_timings(vt, torch, l2, peak_gbs, not args.no_graph)
         line["cpu_baseline"] = cpu_baseline(case)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_profile(args):
+    """A few launches of one kernel family on a small device footprint, for ncu (never a benchmark number)."""
+    import torch
+
+    import paper_2603_05210_b200 as vt
+    torch.cuda.set_device(0)
+    vt.lib()
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    V = inputs.V_LLAMA3
+    if args.profile == "head":
+        d, Vt, M, k = args.d, args.vtrim, args.m or 8, args.k
+        nc = max(2, min(8, -(-400_000_000 // (Vt * d * 2))))            # copies beyond L2 in total, a few hundred MB
+        copies = [(torch.randn((Vt, d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16) for _ in range(nc)]
+        h = torch.randn((M, d), device="cuda", generator=gen).to(torch.bfloat16)
+        d2t = torch.arange(Vt, dtype=torch.int32, device="cuda")
+        ws = vt.new_workspace(vt.vt_workspace_bytes(M, k))
+        for i in range(args.warmup + args.steps):
+            vt.vt_draft_head(h, copies[i % nc], d2t, k, workspace=ws)
+        assert vt.vt_last_status(ws) == vt.VT_OK
+        print(json.dumps({"profile": "head", "d": d, "V_trim": Vt, "M": M, "k": k, "calls": args.warmup + args.steps,
+                          "launches_per_call": vt.vt_last_launch_count()}))
+        return
+    d = args.d
+    W_full = (torch.randn((V, d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16)
+    tokens = inputs.zipf_token_stream(V, 1.05, 10_000_000, 5000)
+    order, _ = inputs.frequency_ranking(tokens, V)
+    keep = to_dev(np.ascontiguousarray(order[:args.vtrim]), torch)
+    tok = [to_dev(tokens, torch) for _ in range(4)]                     # 160 MB of ids: beyond L2
+    cov_ws = torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda")
+    W_trim = vt.vt_compact_head(W_full, keep)
+    for i in range(max(1, args.steps)):
+        vt.vt_compact_head(W_full, keep, out=W_trim)
+        vt.vt_coverage_enqueue(tok[i % 4], keep, V, cov_ws)
+    covered, frac = vt.vt_coverage_result(cov_ws, tokens.size)
+    h3 = torch.randn((8, 3 * d), device="cuda", generator=gen).to(torch.bfloat16)
+    Wf = (torch.randn((d, 3 * d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16)
+    vt.vt_fuse_features(h3, Wf)
+    sel = vt.vt_select_vocab(tok[0], V, d, 2.0 * 3 * d * d + 486.5e6, 0.5, 0.9, 1000, 64000)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile": "aux", "coverage": frac, "k_star": sel["k_star"]}))
 
 
 def bench_config(workload, cold, step, launch, parallelism, calls_per_s):
@@ -371,6 +428,7 @@ def event_us(torch, fn, reps):
     fn()
     pairs = []
     torch.cuda.synchronize()
+    hold_gpu(torch)
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -409,7 +467,7 @@ def once_per_model(vt, torch, W_full, keep, W_trim, tok_dev, tokens, d, V, peak_
         us = event_us(torch, lambda: vt.vt_coverage_enqueue(t, keep, V, cov_ws), 20)
         gbs = 4 * n / us / 1e3
         out["coverage"].append({"tokens": n, "us": round(us, 2), "GBs": round(gbs, 1), "frac": round(gbs / peak_gbs, 4),
-                                "bytes": 4 * n, "what": "bitmap clear + bitmap build + count (3 stream operations), no host read"})
+                                "bytes": 4 * n, "what": "counter clear + one kernel (bitmap built per CTA in shared memory, then the count), no host read"})
     t0 = time.perf_counter()
     for _ in range(10):
         vt.vt_coverage(tok_dev, keep, V, cov_ws)
@@ -456,6 +514,60 @@ def latency_curve(vt, torch, W_full, ranking, case, l2, peak_gbs, use_graph=True
         del copies, W_trim
         torch.cuda.empty_cache()
     return out
+
+
+def fixed_vs_head(vt, torch, curve, d, V, l2, peak_gbs, M=8):
+    """The paper's cost model (Section 2.3, Table 1, Eq. 3) beside what the same split costs on this GPU.
+
+    Eq. 3 predicts the latency reduction of a draft vocabulary of size k from FLOPs: R(k) = 1 - (F_fixed + 2dk) /
+    (F_fixed + 2dV), with F_fixed = fusion + attention + feed-forward (Table 1; the last two are taken as printed).
+    Measured here: the feature-fusion projection (3d -> d, the one fixed component this library runs) and the head at
+    every V_trim of the curve, M draft rows.  R_head_measured(k) = 1 - t_head(k) / t_head(V) is the measured counterpart
+    of Eq. 3 for the head alone (F_fixed = 0); with the measured fusion time added on both sides it is
+    R_fuse_head_measured(k).  On a bandwidth-bound GPU a fixed cost per call flattens both against the FLOPs proxy."""
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    nc = n_copies_for_cold(d * 3 * d * 2, l2, torch.cuda.mem_get_info()[0])
+    Wf = [(torch.randn((d, 3 * d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16) for _ in range(nc)]
+    h3 = torch.randn((M, 3 * d), device="cuda", generator=gen).to(torch.bfloat16)
+    out = torch.empty((M, d), dtype=torch.bfloat16, device="cuda")
+    ws = vt.new_workspace(vt.vt_workspace_bytes(M, 1))
+    i = [0]
+
+    def call():
+        vt.vt_fuse_features(h3, Wf[i[0] % nc], out=out, workspace=ws)
+        i[0] += 1
+
+    for _ in range(10):
+        call()
+    steps = 240
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    hold_gpu(torch)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    assert vt.vt_last_status(ws) == vt.VT_OK
+    t_fuse = e0.elapsed_time(e1) * 1000.0 / steps
+    fuse_bytes = 2 * d * 3 * d + 2 * M * 3 * d + 2 * M * d
+    F_fixed = 2.0 * (3 * d) * d + 436.2e6 + 50.3e6
+    heads = {r["V_trim"]: r["us_per_call"] for r in curve if r["M"] == M}
+    t_full = heads.get(V)
+    rows = []
+    for Vt in sorted(heads):
+        r_eq3 = 1.0 - (F_fixed + 2.0 * d * Vt) / (F_fixed + 2.0 * d * V)
+        row = {"V_trim": Vt, "t_head_us": heads[Vt], "R_eq3": round(r_eq3, 4),
+               "R_eq3_head_only": round(1.0 - Vt / V, 4)}
+        if t_full:
+            row["R_head_measured"] = round(1.0 - heads[Vt] / t_full, 4)
+            row["R_fuse_head_measured"] = round(1.0 - (t_fuse + heads[Vt]) / (t_fuse + t_full), 4)
+        rows.append(row)
+    return {"M": M, "d": d, "t_fuse_us": round(t_fuse, 2), "fuse_bytes": fuse_bytes,
+            "fuse_GBs": round(fuse_bytes / t_fuse / 1e3, 1), "fuse_frac": round(fuse_bytes / t_fuse / 1e3 / peak_gbs, 4),
+            "launch": "eager calls through the binding, back to back, cold copies of W_fuse",
+            "table1_flops": {"fusion": 2.0 * 3 * d * d, "attention": 436.2e6, "feed_forward": 50.3e6, "head_full": 2.0 * d * V},
+            "rows": rows}
 
 
 def config_timings(vt, torch, l2, peak_gbs, use_graph=True):
@@ -595,9 +707,17 @@ def main():
     ap.add_argument("--no-curve", action="store_true")
     ap.add_argument("--m", type=int, default=None, help="draft rows M instead of the workload's 8 (not the headline)")
     ap.add_argument("--no-graph", action="store_true", help="launch every timed call through the binding instead of a CUDA graph")
+    ap.add_argument("--profile", default=None, choices=["head", "aux"],
+                    help="a short run for a profiler instead of the benchmark: 'head' = warm-up + --steps eager head calls on "
+                         "--d/--vtrim/--m/--k (random weights, cold copies); 'aux' = compaction, coverage, selection, fusion once each")
+    ap.add_argument("--d", type=int, default=4096)
+    ap.add_argument("--vtrim", type=int, default=32000)
+    ap.add_argument("--k", type=int, default=8)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.profile:
+        run_profile(args)
     else:
         run_ours(args)
 

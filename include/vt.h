@@ -158,7 +158,9 @@ vt_status vt_draft_head_path(const void* h, const void* W_trim, const int32_t* d
  * target_ids_host / logprobs_host (host [M, k]) are copied back, all on `stream`; the call
  * SYNCHRONISES the stream before returning so the host outputs are valid.  W_trim and d2t
  * stay device-resident (they are model state, not per-step input).  Pinned (page-locked, mapped) output
- * buffers are written by the kernel directly; pageable ones are filled by two copies after it.
+ * buffers are written by the kernel directly; pageable ones are filled by two copies after it.  Which kind a
+ * buffer is is looked up once per buffer address and thread and remembered: keep an output buffer's kind
+ * for as long as its address is passed.
  * workspace: dev, vt_host_workspace_bytes(M, d, k) bytes, initialised with vt_workspace_init. */
 size_t    vt_host_workspace_bytes(int M, int d, int k);
 vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32_t* d2t,

@@ -232,6 +232,26 @@ vt_status vt_draft_head(const void* h, const void* W_trim, const int32_t* d2t, i
 
 static inline size_t up256(size_t b) { return (b + 255) & ~(size_t)255; }
 
+// Device address of a pinned, mapped host buffer (NULL for pageable memory).  A serving loop passes the same
+// two output buffers every step, so each thread remembers the last few answers instead of asking the driver
+// twice per call.  (A buffer that is freed and re-allocated at the same address with another kind of memory
+// would be answered from the cache: the end-to-end call asks that its output buffers stay what they were.)
+static void* mapped_device_pointer(const void* host) {
+    struct Entry { const void* host; void* dev; };
+    static thread_local Entry cache[4] = {};
+    static thread_local int next = 0;
+    for (const Entry& e : cache)
+        if (e.host == host) return e.dev;
+    cudaPointerAttributes at{};
+    void* dev = nullptr;
+    if (cudaPointerGetAttributes(&at, host) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer)
+        dev = at.devicePointer;
+    (void)cudaGetLastError();      // a pageable pointer makes the query fail on some drivers; that is not an error here
+    cache[next] = Entry{host, dev};
+    next = (next + 1) & 3;
+    return dev;
+}
+
 size_t vt_host_workspace_bytes(int M, int d, int k) {
     if (M < 1 || k < 1 || k > VT_MAX_K || d < 8) return 0;
     return ws_total_bytes(M, k) + up256((size_t)M * d * 2) + 2 * up256((size_t)M * k * 4);
@@ -257,15 +277,12 @@ vt_status vt_draft_head_host(const void* h_host, const void* W_trim, const int32
     // addressing): no device-to-host copies.  Pageable outputs go through the staging buffers.
     int32_t* tid_out = tid_dev;
     float* lp_out = lp_dev;
-    cudaPointerAttributes at_tid{}, at_lp{};
-    const bool direct = cudaPointerGetAttributes(&at_tid, target_ids_host) == cudaSuccess &&
-                        cudaPointerGetAttributes(&at_lp, logprobs_host) == cudaSuccess &&
-                        at_tid.type == cudaMemoryTypeHost && at_lp.type == cudaMemoryTypeHost &&
-                        at_tid.devicePointer && at_lp.devicePointer;
-    (void)cudaGetLastError();      // a pageable pointer makes the query fail on some drivers; that is not an error here
+    void* tid_mapped = mapped_device_pointer(target_ids_host);
+    void* lp_mapped = mapped_device_pointer(logprobs_host);
+    const bool direct = tid_mapped != nullptr && lp_mapped != nullptr;
     if (direct) {
-        tid_out = reinterpret_cast<int32_t*>(at_tid.devicePointer);
-        lp_out = reinterpret_cast<float*>(at_lp.devicePointer);
+        tid_out = reinterpret_cast<int32_t*>(tid_mapped);
+        lp_out = reinterpret_cast<float*>(lp_mapped);
     }
     cudaError_t e = cudaMemcpyAsync(h_dev, h_host, (size_t)M * d * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -308,6 +325,7 @@ vt_status vt_coverage_enqueue(const int32_t* token_ids, int64_t N, const int32_t
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < vt_coverage_workspace_bytes(V_full))
         return VT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (coverage_fused_fits(V_full)) return launch_coverage_fused(token_ids, N, keep_ids, V_trim, V_full, workspace, st);
     vt_status r = launch_keep_bitmap(keep_ids, V_trim, V_full, workspace, st);
     if (r != VT_OK) return r;
     return launch_coverage_count(token_ids, N, V_full, workspace, st);

@@ -218,6 +218,97 @@ vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full,
 }
 
 // ------------------------------------------------------------------------------------------
+// The same count in ONE launch, for vocabularies whose bitmap fits in shared memory: every CTA builds the whole
+// membership bitmap for itself from keep_ids (V_trim ids from L2, a few microseconds) and then counts its share of
+// the stream.  No bitmap in global memory, no second kernel: the stream's read is all that touches HBM.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kCoverageThreads) coverage_fused_kernel(
+    const int32_t* __restrict__ token_ids, long long N, const int32_t* __restrict__ keep_ids, int V_trim, int V_full,
+    int bitmap_words, CoverageCounters* counters) {
+    extern __shared__ unsigned int bm_s[];
+    __shared__ unsigned int warp_counts[kCoverageThreads / 32];
+    for (int w = threadIdx.x; w < bitmap_words; w += blockDim.x) bm_s[w] = 0u;
+    __syncthreads();
+    // sixteen ids in flight per thread (four 16-byte loads where keep_ids allows): the whole list costs a few L2
+    // round trips, not one per id
+    auto mark = [&](int v) {
+        if ((unsigned int)v < (unsigned int)V_full) atomicOr(&bm_s[v >> 5], 1u << (v & 31));
+    };
+    const int kvec = (reinterpret_cast<uintptr_t>(keep_ids) & 15) == 0 ? V_trim / 4 : 0;
+    const int4* keep4 = reinterpret_cast<const int4*>(keep_ids);
+    for (int i0 = threadIdx.x; i0 < kvec; i0 += 4 * blockDim.x) {
+        int4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * blockDim.x;
+            v[u] = i < kvec ? __ldg(&keep4[i]) : make_int4(-1, -1, -1, -1);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { mark(v[u].x); mark(v[u].y); mark(v[u].z); mark(v[u].w); }
+    }
+    for (int i = 4 * kvec + threadIdx.x; i < V_trim; i += blockDim.x) mark(__ldg(&keep_ids[i]));
+    __syncthreads();
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(token_ids);
+    long long head = (long long)(((16 - (addr & 15)) & 15) / 4);
+    if (head > N) head = N;
+    const long long nvec = (N - head) / 4;
+    const long long tail_begin = head + nvec * 4;
+    const int4* vec = reinterpret_cast<const int4*>(token_ids + head);
+    unsigned int c = 0;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long gstride = (long long)gridDim.x * blockDim.x;
+    long long i = gtid;
+    for (; i + 3 * gstride < nvec; i += 4 * gstride) {      // four independent 16-byte loads in flight per thread
+        int4 t[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) t[u] = __ldcs(&vec[i + u * gstride]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            c += member(bm_s, t[u].x, V_full) + member(bm_s, t[u].y, V_full) + member(bm_s, t[u].z, V_full) + member(bm_s, t[u].w, V_full);
+    }
+    for (; i < nvec; i += gstride) {
+        const int4 t = __ldcs(&vec[i]);
+        c += member(bm_s, t.x, V_full) + member(bm_s, t.y, V_full) + member(bm_s, t.z, V_full) + member(bm_s, t.w, V_full);
+    }
+    for (long long j = gtid; j < head; j += gstride) c += member(bm_s, token_ids[j], V_full);
+    for (long long j = tail_begin + gtid; j < N; j += gstride) c += member(bm_s, token_ids[j], V_full);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0) warp_counts[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long total = 0;
+        for (int w = 0; w < kCoverageThreads / 32; ++w) total += warp_counts[w];
+        if (total) atomicAdd(&counters->covered, total);
+    }
+}
+
+bool coverage_fused_fits(int V_full) { return coverage_bitmap_words(V_full) * 4 <= kCoverageSmemBitmapMax; }
+
+vt_status launch_coverage_fused(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
+                                void* workspace, cudaStream_t st) {
+    int sms = 0;
+    vt_status rs = device_sm_count(&sms);
+    if (rs != VT_OK) return rs;
+    const size_t words = coverage_bitmap_words(V_full);
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(coverage_fused_kernel), (int)kCoverageSmemBitmapMax, &smem_configured); rc != VT_OK)
+        return rc;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, sizeof(CoverageCounters), st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    // few enough CTAs that re-reading keep_ids once per CTA stays well below the stream's own bytes
+    const long long per_cta = (long long)kCoverageThreads * 4 * 8;
+    const long long by_keep = std::max<long long>(1, (4 * (long long)N) / std::max(1, V_trim));           // CTAs whose keep_ids reads add up to the stream's
+    const long long want = std::min<long long>(((long long)N + per_cta - 1) / per_cta, (long long)sms * 2);
+    const int grid = (int)std::max<long long>(1, std::min<long long>(want, std::max<long long>(8, by_keep)));
+    coverage_fused_kernel<<<grid, kCoverageThreads, words * 4, st>>>(token_ids, N, keep_ids, V_trim, V_full, (int)words,
+                                                                   reinterpret_cast<CoverageCounters*>(workspace));
+    count_launch();
+    e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
 // Coverage without caller-provided scratch: the bitmap and the counters live in a fixed array that is
 // part of the library image on every device that loads it.
 // ------------------------------------------------------------------------------------------

@@ -79,5 +79,9 @@ static_assert(sizeof(CoverageCounters) == 256, "one line");
 inline size_t coverage_bitmap_words(int V_full) { return ((size_t)V_full + 31) / 32; }
 vt_status launch_keep_bitmap(const int32_t* keep_ids, int V_trim, int V_full, void* workspace, cudaStream_t st);
 vt_status launch_coverage_count(const int32_t* token_ids, int64_t N, int V_full, void* workspace, cudaStream_t st);
+// one launch: every CTA builds the bitmap in its shared memory (only where coverage_fused_fits)
+bool coverage_fused_fits(int V_full);
+vt_status launch_coverage_fused(const int32_t* token_ids, int64_t N, const int32_t* keep_ids, int V_trim, int V_full,
+                                void* workspace, cudaStream_t st);
 
 }  // namespace vt

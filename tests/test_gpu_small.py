@@ -76,7 +76,7 @@ def test_coverage_in_two_steps_matches_the_one_call_form(vt, oracle):
     wss = [torch.empty(vt.vt_coverage_workspace_bytes(V), dtype=torch.uint8, device="cuda") for _ in toks]
     for t, ws in zip(devs, wss):
         vt.vt_coverage_enqueue(t, keep_dev, V, ws)
-    assert vt.vt_last_launch_count() == 2
+    assert vt.vt_last_launch_count() == 1            # a bitmap this small is built inside the counting kernel
     for t, ws in zip(toks, wss):
         assert vt.vt_coverage_result(ws, t.size) == oracle.coverage(t, keep, V)
 

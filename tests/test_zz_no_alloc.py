@@ -42,8 +42,8 @@ def test_static_coverage_matches_workspace_coverage_on_two_calls_in_a_row():
     got = vt.vt_coverage_static(tok, second, V)
     free_after, _ = torch.cuda.mem_get_info()
     assert free_after == free_before, (free_before, free_after)
-    assert got == vt.vt_coverage(tok, second, V, ws)
     assert vt.vt_last_launch_count() == 2            # bitmap + count; not added to the previous call's launches
+    assert got == vt.vt_coverage(tok, second, V, ws)
     # a stream that starts off a 16-byte boundary and has a ragged tail (the scalar head / tail path)
     odd = tok[1:300_000 - 2]
     assert odd.data_ptr() % 16 != 0 and odd.numel() % 4 != 0
