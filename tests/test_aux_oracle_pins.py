@@ -77,3 +77,37 @@ def test_fusion_flops_match_table1():
     text = open(__file__.replace("test_aux_oracle_pins.py", "golden/table1_flops.txt")).read()
     assert "100.7" in text
     assert round(2 * (3 * 4096) * 4096 / 1e6, 1) == 100.7
+
+
+def test_tree_selection_vs_repeated_argmax_and_closed_cases():
+    """The tree-step oracle against T passes of "take the best remaining pair" written out with Python floats, on
+    tie-rich scores; with equal parents it reduces to the head's own order; one dominant parent takes every slot."""
+    from oracle import vt_tree_oracle as to
+    rng = np.random.default_rng(9)
+    M, k, T = 6, 5, 11
+    lp = (rng.integers(-6, 0, size=(M, k)) * 0.5).astype(np.float32)
+    lp = -np.sort(-lp, axis=1)                                     # each row descends, like the head's output
+    parent = (rng.integers(-4, 1, size=M) * 0.5).astype(np.float32)
+    tid = rng.integers(0, 1000, size=(M, k)).astype(np.int32)
+    got = to.tree_select(lp, tid, parent, T)
+    score = [[float(np.float32(parent[m]) + np.float32(lp[m, j])) for j in range(k)] for m in range(M)]
+    taken = set()
+    for t in range(T):
+        best = None
+        for m in range(M):
+            for j in range(k):
+                if (m, j) in taken:
+                    continue
+                if best is None or score[m][j] > score[best[0]][best[1]]:      # strict: the first of equals stays
+                    best = (m, j)
+        taken.add(best)
+        assert (got["rows"][t], got["slots"][t]) == best
+        assert got["tokens"][t] == tid[best] and got["scores"][t] == np.float32(score[best[0]][best[1]])
+    # equal parents: row 0's slots first among equals, scores never increase
+    same = to.tree_select(lp, tid, np.zeros(M, dtype=np.float32), M * k)
+    assert np.all(np.diff(same["scores"]) <= 0) and sorted(zip(same["rows"], same["slots"])) == [(m, j) for m in range(M) for j in range(k)]
+    # one parent far above the rest takes its k slots first, in slot order
+    p2 = np.full(M, -100.0, dtype=np.float32)
+    p2[3] = 0.0
+    dom = to.tree_select(lp, tid, p2, k)
+    assert dom["rows"].tolist() == [3] * k and dom["slots"].tolist() == sorted(range(k), key=lambda j: (-lp[3, j], j))
