@@ -191,6 +191,23 @@ vt_status vt_fuse_features(const void* h3, const void* W_fuse, int M, int d_in, 
                            void* fused, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Cross-row candidate selection of a tree-style draft step (Section 1 describes the draft proposing candidate
+ * tokens that the target verifies; the paper gives no formula for expanding several rows at once, so this is the
+ * plain reading, stated here in full):
+ *
+ *   score[m, j] = parent_scores[m] + logprobs[m, j]        one fp32 addition
+ *   the T largest scores over all M * k pairs, in descending order; equal scores by ascending m * k + j
+ *   out_rows[t], out_slots[t] = the pair (m, j);  out_tokens[t] = target_ids[m, j];  out_scores[t] = its score
+ *
+ *   logprobs, target_ids  dev [M, k] (the outputs of vt_draft_head)      parent_scores  dev [M] float
+ *   out_rows, out_slots, out_tokens  dev [T] int32 (out)                 out_scores     dev [T] float (out)
+ * M * k <= 8192, 1 <= T <= M * k.  Asynchronous. */
+vt_status vt_tree_select(const float* logprobs, const int32_t* target_ids, const float* parent_scores,
+                         int M, int k, int T,
+                         int32_t* out_rows, int32_t* out_slots, int32_t* out_tokens, float* out_scores,
+                         void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Coverage of a token stream by the kept set (Eq. 2 with f(v) = occurrences of v in the
  * stream; the "frequency coverage" of Table 4):
  *

@@ -46,6 +46,7 @@ SYMBOLS = {
     "vt_coverage_static": (_i, [_p, _i64, _p, _i, _i, _p, _p, _p]),
     "vt_debug_logits": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p, _i]),
     "vt_fuse_features": (_i, [_p, _p, _i, _i, _i, _p, _p, _sz, _p]),
+    "vt_tree_select": (_i, [_p, _p, _p, _i, _i, _i, _p, _p, _p, _p, _p]),
     "vt_remap": (_i, [_p, _p, _i64, _i, _p, _p]),
     "vt_vocab_maps": (_i, [_p, _i, _i, _p, _p, _p]),
     "vt_last_launch_count": (_i, []),
@@ -298,6 +299,23 @@ def vt_fuse_features(h3: torch.Tensor, W_fuse: torch.Tensor, *, out: torch.Tenso
     _check(lib().vt_fuse_features(h3.data_ptr(), W_fuse.data_ptr(), M, d_in, d_out, out.data_ptr(), workspace.data_ptr(),
                                   workspace.numel(), _stream()), "vt_fuse_features")
     return out
+
+
+def vt_tree_select(logprobs: torch.Tensor, target_ids: torch.Tensor, parent_scores: torch.Tensor, T: int):
+    """The T best (row, slot) pairs by parent score + log-prob: (rows, slots, tokens, scores), each [T]."""
+    M, k = logprobs.shape
+    if logprobs.dtype != torch.float32 or parent_scores.dtype != torch.float32 or not logprobs.is_contiguous():
+        raise ValueError("logprobs and parent_scores must be contiguous float32 CUDA tensors")
+    target_ids = _i32(target_ids, "target_ids")
+    dev = logprobs.device
+    rows = torch.empty(T, dtype=torch.int32, device=dev)
+    slots = torch.empty(T, dtype=torch.int32, device=dev)
+    tokens = torch.empty(T, dtype=torch.int32, device=dev)
+    scores = torch.empty(T, dtype=torch.float32, device=dev)
+    _check(lib().vt_tree_select(logprobs.data_ptr(), target_ids.data_ptr(), parent_scores.data_ptr(), M, k, T,
+                                rows.data_ptr(), slots.data_ptr(), tokens.data_ptr(), scores.data_ptr(), _stream()),
+           "vt_tree_select")
+    return rows, slots, tokens, scores
 
 
 def vt_remap(draft_ids: torch.Tensor, d2t: torch.Tensor) -> torch.Tensor:

@@ -386,6 +386,18 @@ vt_status vt_fuse_features(const void* h3, const void* W_fuse, int M, int d_in, 
     return run_head(c, (cudaStream_t)stream, VT_PATH_AUTO);
 }
 
+vt_status vt_tree_select(const float* logprobs, const int32_t* target_ids, const float* parent_scores, int M, int k, int T,
+                         int32_t* out_rows, int32_t* out_slots, int32_t* out_tokens, float* out_scores, void* stream) {
+    g_launches = 0;
+    if (!logprobs || !target_ids || !parent_scores || !out_rows || !out_tokens || !out_scores || !out_slots) return VT_ERR_NULL;
+    if (M < 1 || k < 1 || T < 1 || (long long)M * k > kTreeSelectMaxPairs || T > M * k) return VT_ERR_SHAPE;
+    if (!aligned(logprobs, 4) || !aligned(target_ids, 4) || !aligned(parent_scores, 4) || !aligned(out_rows, 4) ||
+        !aligned(out_slots, 4) || !aligned(out_tokens, 4) || !aligned(out_scores, 4))
+        return VT_ERR_ALIGN;
+    return launch_tree_select(logprobs, target_ids, parent_scores, M, k, T, out_rows, out_slots, out_tokens, out_scores,
+                              (cudaStream_t)stream);
+}
+
 vt_status vt_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim, int32_t* target_ids,
                    void* stream) {
     g_launches = 0;

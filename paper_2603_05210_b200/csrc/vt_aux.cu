@@ -76,6 +76,54 @@ vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, 
 }
 
 // ------------------------------------------------------------------------------------------
+// Cross-row selection of a tree-style draft step: score[m, j] = parent[m] + logprobs[m, j] (one fp32 addition), the
+// T best of all M * k pairs in descending order, equal scores by ascending flat index.  One CTA: the keys go to
+// shared memory and every pair counts the pairs that beat it - its rank - which is its output position (keys are
+// distinct: they carry the flat index).  n = M * k is a few hundred in practice (at most kTreeMaxPairs).
+// ------------------------------------------------------------------------------------------
+constexpr int kTreeThreads = 512;
+constexpr int kTreeMaxPairs = kTreeSelectMaxPairs;
+
+__global__ void __launch_bounds__(kTreeThreads) tree_select_kernel(const float* __restrict__ logprobs,
+                                                                 const int32_t* __restrict__ target_ids,
+                                                                 const float* __restrict__ parent, int M, int k, int T,
+                                                                 int32_t* __restrict__ out_rows, int32_t* __restrict__ out_slots,
+                                                                 int32_t* __restrict__ out_tokens, float* __restrict__ out_scores) {
+    extern __shared__ unsigned long long keys[];
+    const int n = M * k;
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+        const int m = e / k;
+        keys[e] = make_key(__fadd_rn(parent[m], logprobs[e]), e);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+        const unsigned long long mine = keys[e];
+        int rank = 0;
+        for (int f = 0; f < n; ++f) rank += keys[f] > mine ? 1 : 0;      // every lane reads the same word: a broadcast
+        if (rank < T) {
+            const int m = e / k;
+            out_rows[rank] = m;
+            out_slots[rank] = e - m * k;
+            out_tokens[rank] = target_ids[e];
+            out_scores[rank] = key_logit(mine);
+        }
+    }
+}
+
+vt_status launch_tree_select(const float* logprobs, const int32_t* target_ids, const float* parent, int M, int k, int T,
+                             int32_t* out_rows, int32_t* out_slots, int32_t* out_tokens, float* out_scores, cudaStream_t st) {
+    static std::atomic<unsigned long long> smem_configured{0};
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(tree_select_kernel), kTreeMaxPairs * 8, &smem_configured);
+        rc != VT_OK)
+        return rc;
+    tree_select_kernel<<<1, kTreeThreads, (size_t)M * k * 8, st>>>(logprobs, target_ids, parent, M, k, T, out_rows, out_slots,
+                                                                  out_tokens, out_scores);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// ------------------------------------------------------------------------------------------
 // The two index buffers an EAGLE-3 style draft carries: draft-to-target as offsets
 // (target id = draft index + offset) and target-to-draft as a membership flag per target id.
 // ------------------------------------------------------------------------------------------

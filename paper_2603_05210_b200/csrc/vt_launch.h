@@ -68,6 +68,10 @@ vt_status launch_vocab_maps(const int32_t* keep_ids, int V_trim, int V_full, int
 vt_status launch_remap(const int32_t* draft_ids, const int32_t* d2t, int64_t n, int V_trim,
                        int32_t* target_ids, cudaStream_t st);
 
+constexpr int kTreeSelectMaxPairs = 8192;   // M * k pairs one tree-selection call takes
+vt_status launch_tree_select(const float* logprobs, const int32_t* target_ids, const float* parent, int M, int k, int T,
+                             int32_t* out_rows, int32_t* out_slots, int32_t* out_tokens, float* out_scores, cudaStream_t st);
+
 // Coverage workspace: one 256-byte line of counters, then the membership bitmap.
 struct CoverageCounters {
     unsigned long long covered;
