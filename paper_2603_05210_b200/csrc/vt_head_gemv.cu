@@ -93,17 +93,6 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * S;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * S + 1);
 
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8u * s, 1);
-            mbar_init(bar_empty + 8u * s, 1);
-        }
-        *abort_flag = 0;
-        fence_mbar_init();
-    }
-    for (int i = tid; i < kGemvConsumers * NV * KS; i += blockDim.x) lists[i] = 0ull;
-    __syncthreads();                   // the barriers are initialised: the producer may issue
-
     auto fail = [&]() {
         *abort_flag = 1;
         atomicOr(&p.out.hdr->status, kStatusTimeout);
@@ -116,12 +105,26 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         bulk_g2s(smem_u32(smem) + (uint32_t)s * p.stage_bytes, p.W + (size_t)(row_begin + t * SR) * d, bytes,
                  bar_full + 8u * s);
     };
-    // Nothing above touched global memory.  When the caller has declared W_trim a constant of the model, the
-    // producer starts the first stages before the wait below, while the previous kernel finishes; h, the
-    // workspace and the outputs are only touched after it.
-    const int prefilled = p.early_weights ? min(min(S, ntiles), kGemvPrefill) : 0;
-    if (tid == 0)
-        for (int t = 0; t < prefilled; ++t) issue_tile(t);
+    // The producing thread sets the ring up and starts the stream before it joins the CTA's set-up barrier: the
+    // first bytes take two microseconds to arrive and need nothing else of the set-up.  It waits for the previous
+    // kernel in the stream first - except that, when the caller has declared W_trim a constant of the model, the
+    // first few stages are requested even before that, while the previous kernel finishes.  h, the workspace and
+    // the outputs are only touched after the wait.
+    const int first_fill = min(min(S, ntiles), kGemvPrefill);     // a few stages only: the CTA waits for this thread at the barrier below
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        const int early = p.early_weights ? min(first_fill, kGemvPrefill) : 0;
+        for (int t = 0; t < early; ++t) issue_tile(t);
+        grid_dependency_wait();
+        for (int t = early; t < first_fill; ++t) issue_tile(t);
+    }
+    for (int i = tid; i < kGemvConsumers * NV * KS; i += blockDim.x) lists[i] = 0ull;
+    __syncthreads();                   // the barriers are initialised and the ring is being filled
     grid_dependency_wait();
     if (tid == 0) grid_launch_dependents();
     {   // hidden states of this pass; pad rows (m >= m_count) repeat the last real row and are never read out
@@ -137,8 +140,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            int issued = prefilled;
-            for (int t = prefilled; t < ntiles; ++t) {
+            int issued = first_fill;
+            for (int t = first_fill; t < ntiles; ++t) {
                 const int s = t % S, n = t / S;
                 if (n > 0 && !mbar_wait(bar_empty + 8u * s, (uint32_t)(n - 1) & 1u)) { fail(); break; }
                 if (*abort_flag) break;
