@@ -291,3 +291,10 @@ def test_host_buffer_entry_point(vt, oracle, pinned):
         tid.fill_(-7)
         vt.vt_draft_head_host(h_host, Wd, d2td, k, tid, lp, ws)
         parity.check_head({"target_ids": tid.numpy().copy(), "logprobs": lp.numpy().copy()}, ora, d2t, k)
+    # new hidden states in the SAME host buffer: the next call must see them (nothing of the old ones may be cached)
+    for seed in (14, 15):
+        h2 = inputs.hidden_states_bf16(M, d, seed)
+        h_host.copy_(torch.from_numpy(h2.view(np.int16).copy()))
+        vt.vt_draft_head_host(h_host, Wd, d2td, k, tid, lp, ws)
+        parity.check_head({"target_ids": tid.numpy().copy(), "logprobs": lp.numpy().copy()},
+                          oracle.draft_head(h2, W, d2t, k, want_logits=True), d2t, k)
