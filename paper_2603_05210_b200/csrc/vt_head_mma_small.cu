@@ -40,7 +40,9 @@ namespace vt {
 
 constexpr int kSmMaxEpiWarps = 16;            // warps 0-7, or 0-15 when there are more than 8 draft rows; 0-3 also read TMEM
 constexpr int kSmThreads = (kSmMaxEpiWarps + 2) * 32;     // at most: the epilogue warps, then the producer, then the MMA issuer
-constexpr int kSmMaxM = 128;                  // draft rows per launch <= MMA N <= 128
+constexpr int kSmMaxM = 128;                  // draft rows per launch = MMA N
+constexpr int kSmMaxMChunked = 256;           // ... when a CTA has one tile and the thread-per-row epilogue takes it 64 draft rows at a time
+constexpr int kChunkRows = 64;
 constexpr int kLgRows = 32;                   // draft rows whose tile logits shared memory holds at a time
 constexpr int kSmMaxStages = 32;
 constexpr int kLgPitch = 132;                 // floats between draft rows of the tile's logits in shared memory
@@ -49,12 +51,13 @@ constexpr int kSmCand = 128 + VT_MAX_K;       // candidate keys per epilogue war
 
 struct SmallParams {
     HeadOut out;
-    int M;                    // draft rows of this launch, <= kSmMaxM
+    int M;                    // draft rows of this launch, <= kSmMaxM (<= kSmMaxMChunked with chunked thread-per-row)
     int m_begin;              // first of them among the call's draft rows
     int merge_in_kernel;      // 1: one draft row per epilogue warp, merged by the last warp to publish it; 0: a merge kernel follows
     int n_epi;                // epilogue warps: 8, or 16 when M > 8 with the warp-per-row epilogue; the block has
                               // two more (producer, MMA issuer)
-    int lg_rows;              // draft rows whose tile logits shared memory holds at a time: kLgRows, or all with thread-per-row
+    int lg_rows;              // draft rows whose tile logits shared memory holds at a time: kLgRows with warp-per-row;
+                              // with thread-per-row all of them, or 64 at a time when the CTA has a single tile
     uint32_t scratch_stride;  // bytes of one epilogue warp's candidate buffer: (128 + k) keys
     int N;                    // MMA N: M rounded up to a multiple of 16
     int h_resident;           // 1: h sits in shared memory for the whole kernel (h_off); 0: one block per k-block in the ring
@@ -98,7 +101,10 @@ __device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.syn
 
 // KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue for more than 16 draft rows, with a
 // register list of KR >= k entries per thread.
-template <int KR>
+// PAIR: launched as clusters of two CTAs that share one MMA of 256 lanes (chunked thread-per-row only, one tile per
+// CTA): each CTA streams its own vocabulary rows and HALF of every k-block of h, so h crosses from L2 to the SMs
+// 74 times instead of 148 - with 128 and more draft rows that traffic, not the weight stream, was the bound.
+template <int KR, bool PAIR>
 __global__ void __launch_bounds__(kSmThreads, 1)
 head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH,
                       const SmallParams p) {
@@ -116,6 +122,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     const int nrows = row_end - row_begin;
     const int ntiles = (nrows + TH - 1) / TH;
     const int h_part = (nk + kHParts - 1) / kHParts;          // k-blocks per part of h
+    const uint32_t pair_rank = PAIR ? cluster_cta_rank() : 0u;
+    const bool leader = pair_rank == 0u;                      // issues the MMAs (always true without pairs)
 
     float* lg = reinterpret_cast<float*>(smem + p.lg_off);                                  // [M][kLgPitch]
     unsigned long long* lists = reinterpret_cast<unsigned long long*>(smem + p.list_off);   // [M][k]
@@ -162,13 +170,20 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         for (int i = tid; i < 256 * KF; i += blockDim.x)
             reinterpret_cast<uint32_t*>(smem + p.h_off + (uint32_t)nk * p.h_blk)[i] = 0u;
     if (warp == mma_warp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (PAIR) {     // the same warp of both CTAs
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     fence_proxy_async();          // the zeroed pad is read by the tensor core (async proxy)
     tc_fence_before();
-    __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();      // the other CTA's barriers are initialised before anything arrives on them
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above touched only shared memory, tensor memory and kernel parameters, so under programmatic
@@ -191,12 +206,24 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             const int total = ntiles * spt;                 // ring stages of this CTA, in issue order
             const uint64_t stream_once = l2_policy_evict_first();
             const uint32_t h_tx = p.h_resident ? 0u : p.h_blk;
+            const int h_row0 = p.m_begin + (PAIR ? (int)pair_rank * (p.N >> 1) : 0);     // a pair's CTAs hold N/2 rows of h each
             // stage q of the CTA's sequence into ring slot s: the weight boxes and the matching blocks of h
             auto issue = [&](int q, int s) {
                 const int t = q / spt, ks = (q - t * spt) * kbs;
                 const int row0 = row_begin + t * TH;
                 const int nb = min(kbs, nsb - ks);
                 const uint32_t bar = bar_full + 8u * s;
+                if constexpr (PAIR) {
+                    // both CTAs' bytes are counted on the leader's barrier, which its producer arms
+                    if (leader) mbar_arrive_expect_tx(bar, 2u * (uint32_t)nb * (p.w_tx + h_tx));
+                    const uint32_t lbar = cluster_map_shared(bar, 0u);
+                    for (int kb = 0; kb < nb; ++kb) {
+                        const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
+                        tma_load_2d_pair_hint(dst, &tmW, (ks + kb) * kBoxK, row0, lbar, stream_once);
+                        tma_load_2d_pair(dst + p.slot_bytes, &tmH, (ks + kb) * kBoxK, h_row0, lbar);
+                    }
+                    return;
+                }
                 mbar_arrive_expect_tx(bar, (uint32_t)nb * (uint32_t)KF * (p.w_tx + h_tx));
                 for (int kb = 0; kb < nb; ++kb) {
                     const uint32_t dst = base + (uint32_t)s * p.stage_bytes + (uint32_t)kb * p.blk_bytes;
@@ -207,7 +234,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (!p.h_resident)                // the matching k-blocks of h, one block after the other behind the weights
                         for (int g = 0; g < KF; ++g)
                             tma_load_2d(dst + p.slot_bytes + (uint32_t)g * p.h_blk, &tmH, ((ks + kb) * KF + g) * kBoxK,
-                                        p.m_begin, bar);
+                                        h_row0, bar);
                 }
             };
             int s = 0, issued = 0;
@@ -219,15 +246,17 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 ++issued;
                 if (++s == S) { s = 0; ++wrap; }
             }
-            if (*abort_flag) {   // let copies in flight land before the CTA gives its shared memory back
+            if (*abort_flag && leader) {   // let copies in flight land before the CTA gives its shared memory back
+                // (in a pair the leader's barriers count both CTAs' copies, and the other CTA leaves only after
+                // the leader has passed this point: the cluster-wide barrier at the end)
                 const unsigned long long deadline = global_timer_ns() + kWaitLimitNs;
                 for (int i = max(0, issued - S); i < issued; ++i)
                     (void)mbar_wait_until(bar_full + 8u * (i % S), (uint32_t)(i / S) & 1u, deadline);
             }
         }
     } else if (warp == mma_warp) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (in a pair: the leader's)
+        if (lane == 0 && leader) {
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -257,18 +286,31 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         const uint64_t b_desc = p.h_resident ? h_desc0 + (uint64_t)((uint32_t)((ks + kb) * KF) * h_units)
                                                              : a_desc + slot_units;
                         // 16 bf16 = 32 bytes = 2 descriptor address units per MMA along K
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
-                        tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                        if constexpr (PAIR) {
+                            tc_mma_bf16_pair(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
+                            tc_mma_bf16_pair(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
+                            tc_mma_bf16_pair(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
+                            tc_mma_bf16_pair(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                        } else {
+                            tc_mma_bf16(d_tmem, a_desc, b_desc, p.idesc, (ks | kb) != 0);
+                            tc_mma_bf16(d_tmem, a_desc + 2u, b_desc + 2u, p.idesc, 1u);
+                            tc_mma_bf16(d_tmem, a_desc + 4u, b_desc + 4u, p.idesc, 1u);
+                            tc_mma_bf16(d_tmem, a_desc + 6u, b_desc + 6u, p.idesc, 1u);
+                        }
                     }
-                    tc_commit(bar_empty + 8u * s);
+                    // the stage is free (in both CTAs of a pair) once these MMAs have read it
+                    if constexpr (PAIR) tc_commit_pair_both(bar_empty + 8u * s);
+                    else tc_commit(bar_empty + 8u * s);
                     if (++s == S) { s = 0; phase ^= 1u; }
                 }
-                if (ok) tc_commit(bar_accf + 8u * buf);
+                if (ok) {
+                    if constexpr (PAIR) tc_commit_pair_both(bar_accf + 8u * buf);
+                    else tc_commit(bar_accf + 8u * buf);
+                }
             }
             if (*abort_flag) {   // every MMA issued so far must retire before TMEM is freed
-                tc_commit(bar_drain);
+                if constexpr (PAIR) tc_commit_pair(bar_drain);
+                else tc_commit(bar_drain);
                 (void)mbar_wait(bar_drain, 0u);
             }
         }
@@ -285,134 +327,158 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         // assignment and fold the same logits into the rows' running (max, sum-exp): the two kinds of work use
         // different pipes (compare/select against multiply-add and exp2) and hide each other's latencies.
         constexpr int KL = KR > 0 ? KR : 1;
+        // A CTA with a single tile takes its draft rows CH = 64 at a time and writes their records right away:
+        // shared memory then holds 64 rows of logits instead of all of them and the ring gets the difference.
         const bool scanner = warp < 4;
         const int w4 = warp & 3;
-        const int RG = (M + 31) >> 5;                                  // groups of 32 draft rows: 1 .. 4
+        const int CH = p.lg_rows;                                      // draft rows per pass of the epilogue
+        const int nch = (M + CH - 1) / CH;                             // 1 unless the CTA has a single tile
+        const int RG = (min(M, CH) + 31) >> 5;                         // groups of 32 draft rows: 1 .. 4
         const int Q = RG == 1 ? 4 : RG == 2 ? 2 : 1;                   // column ranges a row is split into
         const int rg = w4 % RG, part = w4 / RG;
         const bool works = part < Q;                                   // warp-uniform
         const int m_own = rg * 32 + lane;                              // the thread's draft row of this pass
         const int xs = RG * 32;
-        const float* rowp = lg + (size_t)min(m_own, M - 1) * kLgPitch;     // lanes past the last row re-read it and keep nothing
         float v[KL];
         int ix[KL];
 #pragma unroll
         for (int j = 0; j < KL; ++j) { v[j] = -INFINITY; ix[j] = -1; }
         float mx = -INFINITY, ssum = 0.0f;
         int seen = 0;                                                  // logits this thread has scanned (the same in every lane of a warp)
+        unsigned long long* xl = reinterpret_cast<unsigned long long*>(lg);      // [(part * RG * 32 + row) * (KL + 1)], see below
         for (int t = 0; t < ntiles; ++t) {
             const int buf = t & 1;
             const int row0 = row_begin + t * TH;
             const int nv = min(TH, row_end - row0);
+            bool got = false;
             if (scanner) {
                 // warp-uniform decisions: tcgen05.ld needs the whole warp
-                bool got = false;
                 if (!__any_sync(0xFFFFFFFFu, *abort_flag != 0)) {
                     got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_accf + 8u * buf, (uint32_t)(t >> 1) & 1u));
                     if (!got) fail();
                 }
-                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
-                if (KF > 1) {
-                    // Folded k-blocks: this warp's lanes are k-group g of tile rows r0 + lane, and columns
-                    // NG*g .. NG*g + NG - 1 of the accumulator are their partial logits for the draft rows.
-                    const int SR = 128 / KF, NG = p.NG, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
-                    float* partial = reinterpret_cast<float*>(smem + p.part_off);
-                    if (got) {
-                        tc_fence_after();
-                        for (int c0 = 0; c0 < NG; c0 += 16) {
-                            uint32_t u[16];
-                            tc_ld16(taddr + (uint32_t)(NG * g + c0), u);
-                            tc_wait_ld();
+            }
+            for (int ch = 0; ch < nch; ++ch) {
+                const int m0 = ch * CH, Mc = min(CH, M - m0);          // this pass: draft rows m0 .. m0 + Mc - 1 of the launch
+                const float* rowp = lg + (size_t)min(m_own, Mc - 1) * kLgPitch;   // lanes past the last row re-read it and keep nothing
+                if (scanner) {
+                    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
+                    if (KF > 1) {
+                        // Folded k-blocks (never with several passes): this warp's lanes are k-group g of tile rows
+                        // r0 + lane, and columns NG*g .. NG*g + NG - 1 of the accumulator are their partial logits
+                        // for the draft rows.
+                        const int SR = 128 / KF, NG = p.NG, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
+                        float* partial = reinterpret_cast<float*>(smem + p.part_off);
+                        if (got) {
+                            tc_fence_after();
+                            for (int c0 = 0; c0 < NG; c0 += 16) {
+                                uint32_t u[16];
+                                tc_ld16(taddr + (uint32_t)(NG * g + c0), u);
+                                tc_wait_ld();
 #pragma unroll
-                            for (int m = 0; m < 16; ++m) partial[(g * NG + c0 + m) * 64 + r] = __uint_as_float(u[m]);
+                                for (int m = 0; m < 16; ++m) partial[(g * NG + c0 + m) * 64 + r] = __uint_as_float(u[m]);
+                            }
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
                         }
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
-                    }
-                    reader_barrier();                              // all four readers' partial sums are in place
-                    for (int e = tid; e < M * SR; e += 128) {
-                        const int m = e / SR, rr = e - m * SR;
-                        if (rr >= nv) continue;
-                        float sum = 0.0f;
-                        for (int gg = 0; gg < KF; ++gg) sum += partial[(gg * p.NG + m) * 64 + rr];
-                        lg[m * kLgPitch + rr] = sum;
-                        if (wants_logits(p.out)) store_logit(p.out, p.m_begin + m, row0 + rr, sum);
-                    }
-                } else if (got) {
-                    const int i = warp * 32 + lane;                // TMEM lane = vocabulary row of the tile
-                    tc_fence_after();
-                    for (int c1 = 0; c1 < M; c1 += 16) {           // 16 draft rows per load
-                        uint32_t u[16];
-                        tc_ld16(taddr + (uint32_t)c1, u);
-                        tc_wait_ld();
-                        if (i < nv) {
-#pragma unroll
-                            for (int m = 0; m < 16; ++m)
-                                if (c1 + m < M) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(u[m]);
-                            if (wants_logits(p.out)) {
+                        reader_barrier();                              // all four readers' partial sums are in place
+                        for (int e = tid; e < M * SR; e += 128) {
+                            const int m = e / SR, rr = e - m * SR;
+                            if (rr >= nv) continue;
+                            float sum = 0.0f;
+                            for (int gg = 0; gg < KF; ++gg) sum += partial[(gg * p.NG + m) * 64 + rr];
+                            lg[m * kLgPitch + rr] = sum;
+                            if (wants_logits(p.out)) store_logit(p.out, p.m_begin + m, row0 + rr, sum);
+                        }
+                    } else if (got) {
+                        const int i = warp * 32 + lane;                // TMEM lane = vocabulary row of the tile
+                        if (ch == 0) tc_fence_after();
+                        for (int c1 = 0; c1 < Mc; c1 += 16) {          // 16 draft rows per load
+                            uint32_t u[16];
+                            tc_ld16(taddr + (uint32_t)(m0 + c1), u);
+                            tc_wait_ld();
+                            if (i < nv) {
 #pragma unroll
                                 for (int m = 0; m < 16; ++m)
-                                    if (c1 + m < M) store_logit(p.out, p.m_begin + c1 + m, row0 + i, __uint_as_float(u[m]));
+                                    if (c1 + m < Mc) lg[(c1 + m) * kLgPitch + i] = __uint_as_float(u[m]);
+                                if (wants_logits(p.out)) {
+#pragma unroll
+                                    for (int m = 0; m < 16; ++m)
+                                        if (c1 + m < Mc)
+                                            store_logit(p.out, p.m_begin + m0 + c1 + m, row0 + i, __uint_as_float(u[m]));
+                                }
                             }
                         }
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
-                }
-            }
-            epi_barrier(256);                                      // the tile's logits are in shared memory
-            // ---- the thread's own columns [cb, ce) of its draft row.  After a wait ran out the buffer holds the
-            // previous tile again: whatever is computed from it belongs to a call that reports the time-out.
-            const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
-            const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
-            if (works && n > 0 && !p.out.store_only) {
-                if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + tid);
-                else row_scan_lse(rowp, cb, ce, mx, ssum);
-            }
-            seen += max(n, 0);
-            epi_barrier(256);                                      // the buffer may be overwritten
-        }
-        // ---- the rows' records: best k keys and (max, sum-exp).  The logits buffer is free now: it takes every
-        // thread's list (or sums); the range-0 scanner of a row merges its column ranges and writes the record.
-        unsigned long long* xl = reinterpret_cast<unsigned long long*>(lg);      // [(part * RG * 32 + row) * (KL + 1)]
-        if (works) {
-            unsigned long long* mine = xl + (size_t)(part * xs + m_own) * (KL + 1);
-            if (scanner) {
-#pragma unroll
-                for (int j = 0; j < KL; ++j) mine[j] = ix[j] >= 0 ? make_key(v[j], ix[j]) : 0ull;
-            } else {
-                mine[KL] = pack_ms(mx, ssum);
-            }
-        }
-        epi_barrier(256);
-        if (scanner && part == 0 && m_own < M && !p.out.store_only) {
-            const int row = p.m_begin + m_own;                                 // among the call's draft rows
-            // Q sorted lists: the best remaining key is the largest head, k times
-            int pos[4] = {0, 0, 0, 0};
-            for (int j = 0; j < k; ++j) {
-                unsigned long long best = 0ull;
-                int bq = 0;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (q < Q && pos[q] < KL) {
-                        const unsigned long long key = xl[(size_t)(q * xs + m_own) * (KL + 1) + pos[q]];
-                        if (key > best) { best = key; bq = q; }
+                        if (ch == nch - 1) {                           // the accumulator is read out
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                        }
                     }
                 }
+                epi_barrier(256);                                      // the pass's logits are in shared memory
+                // ---- the thread's own columns [cb, ce) of its draft row.  After a wait ran out the buffer holds
+                // older logits: whatever is computed from them belongs to a call that reports the time-out.
+                const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
+                const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
+                if (works && n > 0 && !p.out.store_only) {
+                    if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + tid);
+                    else row_scan_lse(rowp, cb, ce, mx, ssum);
+                }
+                seen += max(n, 0);
+                epi_barrier(256);                                      // the buffer may be overwritten
+                if (nch == 1 && t + 1 < ntiles) continue;              // lists and sums carry over to the next tile
+                // ---- the rows' records: best k keys and (max, sum-exp).  The logits buffer is free now: it takes
+                // every thread's list (or sums); the range-0 scanner of a row merges its column ranges and writes
+                // the record.
+                if (works) {
+                    unsigned long long* mine = xl + (size_t)(part * xs + m_own) * (KL + 1);
+                    if (scanner) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) pos[q] += (q == bq && best != 0ull) ? 1 : 0;
-                VT_ROW_KEYS(p.out, row, j)[cta] = best;
+                        for (int j = 0; j < KL; ++j) mine[j] = ix[j] >= 0 ? make_key(v[j], ix[j]) : 0ull;
+                    } else {
+                        mine[KL] = pack_ms(mx, ssum);
+                    }
+                }
+                epi_barrier(256);
+                if (scanner && part == 0 && m_own < Mc && !p.out.store_only) {
+                    const int row = p.m_begin + m0 + m_own;                    // among the call's draft rows
+                    // Q sorted lists: the best remaining key is the largest head, k times
+                    int pos[4] = {0, 0, 0, 0};
+                    for (int j = 0; j < k; ++j) {
+                        unsigned long long best = 0ull;
+                        int bq = 0;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (q < Q && pos[q] < KL) {
+                                const unsigned long long key = xl[(size_t)(q * xs + m_own) * (KL + 1) + pos[q]];
+                                if (key > best) { best = key; bq = q; }
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) pos[q] += (q == bq && best != 0ull) ? 1 : 0;
+                        VT_ROW_KEYS(p.out, row, j)[cta] = best;
+                    }
+                    float cmx = -INFINITY;
+                    for (int q = 0; q < Q; ++q) cmx = fmaxf(cmx, unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]).x);
+                    float cs = 0.0f;
+                    for (int q = 0; q < Q; ++q) {
+                        const float2 ms = unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]);
+                        if (ms.y > 0.0f) cs += ms.y * __expf(ms.x - cmx);
+                    }
+                    VT_ROW_MS(p.out, row)[cta] = pack_ms(cmx, cs);
+                }
+                if (ch + 1 < nch) {
+                    // the next pass starts from empty lists, once the exchange buffer has been read
+#pragma unroll
+                    for (int j = 0; j < KL; ++j) { v[j] = -INFINITY; ix[j] = -1; }
+                    mx = -INFINITY;
+                    ssum = 0.0f;
+                    seen = 0;
+                    epi_barrier(256);
+                }
             }
-            float cmx = -INFINITY;
-            for (int q = 0; q < Q; ++q) cmx = fmaxf(cmx, unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]).x);
-            float cs = 0.0f;
-            for (int q = 0; q < Q; ++q) {
-                const float2 ms = unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]);
-                if (ms.y > 0.0f) cs += ms.y * __expf(ms.x - cmx);
-            }
-            VT_ROW_MS(p.out, row)[cta] = pack_ms(cmx, cs);
         }
     } else if (KR == 0 && warp < p.n_epi) {
         // ------------------------------------------------------------------ epilogue warps
@@ -553,16 +619,21 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     }
 
     tc_fence_before();
-    __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();      // neither CTA leaves while the other's MMAs or arrivals may still reach it
+    else __syncthreads();
     tc_fence_after();
-    if (warp == mma_warp)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    if (warp == mma_warp) {
+        if constexpr (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    }
 }
 
 // ------------------------------------------------------------------------------------------ host
 // Tile geometry and shared-memory layout for a shape; false if it does not fit.
-static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, int* list_regs) {
-    if (M < 1 || M > kSmMaxM) return false;
+static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, SmallParams* p, int* list_regs, bool* pair_out) {
+    if (M < 1 || M > kSmMaxMChunked) return false;
     const int R = (Vt + grid - 1) / grid;                    // most rows a CTA owns
     const int nt = (R + 127) / 128;
     // More than 16 draft rows: one thread per draft row, as long as a register list holds k entries.  With four
@@ -570,13 +641,21 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, in
     // and leaves more shared memory to the ring (measured at V_trim = 128256: 180 against 194 us).
     const int KR = (M > 16 && !(M <= 64 && nt >= 4)) ? topk_list_regs(k) : 0;
     *list_regs = KR;
+    // One tile per CTA and more than 64 draft rows: the epilogue takes the tile 64 draft rows at a time (nothing
+    // carries over to a next tile), which frees 34 KB and more for the ring and lets one launch take 256 draft rows.
+    const bool chunked = KR > 0 && nt == 1 && M > kChunkRows;
+    if (M > kSmMaxM && !chunked) return false;
+    // ... and then two CTAs share each MMA, each fetching half of h
+    const bool pair = chunked && pairs_ok && (grid & 1) == 0;
+    *pair_out = pair;
+    const int n_round = pair ? 32 : 16;                      // MMA N: a pair's CTAs hold whole 16-row blocks of h each
     p->M = M;
     p->d = d;
     p->nk = (d + kBoxK - 1) / kBoxK;
     p->TH = (R + nt - 1) / nt;
     p->w_tx = (uint32_t)p->TH * 128u;
-    p->h_blk = M <= 8 ? 1024u : (uint32_t)(((M + 15) / 16) * 16) * 128u;
-    p->lg_rows = KR > 0 ? ((M + 15) / 16) * 16 : std::min(M, kLgRows);
+    p->h_blk = M <= 8 ? 1024u : (uint32_t)(((M + n_round - 1) / n_round) * n_round) * (pair ? 64u : 128u);
+    p->lg_rows = chunked ? kChunkRows : KR > 0 ? ((M + 15) / 16) * 16 : std::min(M, kLgRows);
     // thread-per-row: all of the tile's draft rows at once, and room for the column ranges' lists at the end
     const size_t lg_bytes = KR > 0 ? (std::max((size_t)p->lg_rows * kLgPitch * 4, (size_t)128 * (KR + 1) * 8) + 127) & ~(size_t)127
                                    : ((size_t)p->lg_rows * kLgPitch * 4 + 127) & ~(size_t)127;
@@ -600,13 +679,14 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, in
         // rows, M = 48 and 64 at 28), so there it is four or nothing
         if (!resident && (p->G < 4 || 4 * p->NG > 128)) p->G = 1;
         p->nsb = (p->nk + p->G - 1) / p->G;
-        p->N = p->G > 1 ? p->NG * p->G : ((M + 15) / 16) * 16;
+        p->N = p->G > 1 ? p->NG * p->G : ((M + n_round - 1) / n_round) * n_round;
         p->sub_bytes = (uint32_t)(128 / p->G) * 128u;
         p->slot_bytes = p->G > 1 ? 16384u : (uint32_t)((p->TH + 7) / 8) * 1024u;
         p->tmem_cols = 32;
         while (p->tmem_cols < 2u * (uint32_t)p->N) p->tmem_cols *= 2;
         // instruction descriptor: D fp32, A and B bf16, both K-major, N, M = 128
-        p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // (a pair's MMA: M = 256, 128 lanes in either CTA)
+        p->idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p->N >> 3) << 17) | ((uint32_t)((pair ? 256 : 128) >> 4) << 24);
         const size_t part_bytes = p->G > 1 ? (size_t)p->G * p->NG * 64 * 4 : 0;
         // + zeros for what the last MMA step reads past h: rows 8-15 of an unfolded step, whole k-blocks of a folded one
         const size_t h_bytes = resident ? (size_t)p->nk * p->h_blk + 1024 * (size_t)p->G : 0;
@@ -645,16 +725,48 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, SmallParams* p, in
     return false;
 }
 
-template <int KR>
+template <int KR, bool PAIR>
 static vt_status launch_small(const CUtensorMap& tmW, const CUtensorMap& tmH, const SmallParams& p, int grid, cudaStream_t st) {
     static std::atomic<unsigned long long> smem_configured{0};
-    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel<KR>), kMaxDynSmem, &smem_configured);
+    if (vt_status rc = ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel<KR, PAIR>), kMaxDynSmem, &smem_configured);
         rc != VT_OK)
         return rc;
-    cudaError_t e = launch_pdl(head_mma_small_kernel<KR>, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
+    cudaError_t e = PAIR ? launch_pdl_cluster2(head_mma_small_kernel<KR, PAIR>, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p)
+                         : launch_pdl(head_mma_small_kernel<KR, PAIR>, grid, (p.n_epi + 2) * 32, p.total_smem, st, tmW, tmH, p);
     count_launch();
     if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? VT_OK : cuda_fail(e);
+}
+
+// Whether `grid` CTAs of the pair kernel with the largest shared-memory request can all be resident as clusters of
+// two (asked once per process; the answer does not depend on the list length).
+static bool pairs_schedulable(int grid) {
+    static std::atomic<int> cached{-1};          // most clusters the device holds at once
+    int n = cached.load(std::memory_order_acquire);
+    if (n < 0) {
+        static std::atomic<unsigned long long> smem_configured{0};
+        if (ensure_max_dyn_smem(reinterpret_cast<const void*>(head_mma_small_kernel<10, true>), kMaxDynSmem, &smem_configured) != VT_OK)
+            return false;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3((unsigned)(10 * 32));
+        cfg.dynamicSmemBytes = kMaxDynSmem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, head_mma_small_kernel<10, true>, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            clusters = 0;
+        }
+        n = clusters;
+        cached.store(n, std::memory_order_release);
+    }
+    return 2 * n >= grid;
 }
 
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_out) {
@@ -663,31 +775,47 @@ vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid_ou
     if (r != VT_OK) return r;
     const int grid = head_grid(sms, c.Vt, 16);
     *grid_out = grid;
-    // every pass of kSmMaxM draft rows must fit before anything is launched
-    int KR = 0;
-    for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {
+    const bool pairs_ok = c.M > kChunkRows && (grid & 1) == 0 && pairs_schedulable(grid);
+    // draft rows per pass: 256 where the plan takes them (one tile per CTA, thread-per-row), else 128
+    int KR = 0, pass = kSmMaxM;
+    bool pair = false;
+    if (c.M > kSmMaxM) {
         SmallParams q{};
-        if (!small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &q, &KR)) return VT_ERR_UNSUPPORTED;
+        if (small_plan(std::min(kSmMaxMChunked, c.M), c.d, c.Vt, c.out.k, grid, pairs_ok, &q, &KR, &pair)) pass = kSmMaxMChunked;
+    }
+    // every pass must fit before anything is launched
+    for (int m0 = 0; m0 < c.M; m0 += pass) {
+        SmallParams q{};
+        if (!small_plan(std::min(pass, c.M - m0), c.d, c.Vt, c.out.k, grid, pairs_ok, &q, &KR, &pair)) return VT_ERR_UNSUPPORTED;
     }
     bool merge_after = false;
-    for (int m0 = 0; m0 < c.M; m0 += kSmMaxM) {        // each pass streams the weights once for its draft rows
+    for (int m0 = 0; m0 < c.M; m0 += pass) {           // each pass streams the weights once for its draft rows
         SmallParams p{};
-        small_plan(std::min(kSmMaxM, c.M - m0), c.d, c.Vt, c.out.k, grid, &p, &KR);
+        small_plan(std::min(pass, c.M - m0), c.d, c.Vt, c.out.k, grid, pairs_ok, &p, &KR, &pair);
         p.out = c.out;
         p.m_begin = m0;
-        if (c.M > kSmMaxM) p.merge_in_kernel = 0;       // row tickets serve single-pass calls only
+        if (c.M > pass) p.merge_in_kernel = 0;          // row tickets serve single-pass calls only
         merge_after = !p.merge_in_kernel;
         CUtensorMap tmW, tmH;
         r = make_tensor_map_bf16(&tmW, c.W, c.Vt, c.d, p.TH);
         if (r != VT_OK) return r;
         r = make_tensor_map_bf16(&tmH, c.h, c.M, c.d, (int)(p.h_blk / 128u));
         if (r != VT_OK) return r;
-        switch (KR) {
-            case 4: r = launch_small<4>(tmW, tmH, p, grid, st); break;
-            case 8: r = launch_small<8>(tmW, tmH, p, grid, st); break;
-            case 10: r = launch_small<10>(tmW, tmH, p, grid, st); break;
-            case 16: r = launch_small<16>(tmW, tmH, p, grid, st); break;
-            default: r = launch_small<0>(tmW, tmH, p, grid, st); break;
+        if (pair) {
+            switch (KR) {
+                case 4: r = launch_small<4, true>(tmW, tmH, p, grid, st); break;
+                case 8: r = launch_small<8, true>(tmW, tmH, p, grid, st); break;
+                case 10: r = launch_small<10, true>(tmW, tmH, p, grid, st); break;
+                default: r = launch_small<16, true>(tmW, tmH, p, grid, st); break;
+            }
+        } else {
+            switch (KR) {
+                case 4: r = launch_small<4, false>(tmW, tmH, p, grid, st); break;
+                case 8: r = launch_small<8, false>(tmW, tmH, p, grid, st); break;
+                case 10: r = launch_small<10, false>(tmW, tmH, p, grid, st); break;
+                case 16: r = launch_small<16, false>(tmW, tmH, p, grid, st); break;
+                default: r = launch_small<0, false>(tmW, tmH, p, grid, st); break;
+            }
         }
         if (r != VT_OK) return r;
     }

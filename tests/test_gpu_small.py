@@ -167,7 +167,12 @@ HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8)
                (4, 5120, 700, 8), (64, 512, 333, 10), (5, 200, 2000, 33), (1, 4096, 13264, 1),
                (16, 256, 40000, 10), (7, 64, 60001, 64), (12, 4096, 3000, 8), (2, 8192, 600, 5),
                (33, 1024, 20000, 10), (64, 4096, 2500, 8), (48, 2048, 9000, 16), (8, 16384, 400, 4),
-               (100, 2048, 30000, 10), (128, 512, 1000, 8), (257, 256, 20000, 3)]
+               (100, 2048, 30000, 10), (128, 512, 1000, 8), (257, 256, 20000, 3),
+               # more than 64 draft rows and one tile per CTA: the tensor-core kernel takes the tile 64 draft rows at a
+               # time, CTA pairs share each MMA, one launch holds up to 256 draft rows
+               (65, 256, 5000, 10), (100, 1024, 16384, 10), (128, 512, 2368, 8), (129, 512, 18944, 4),
+               (200, 2048, 9000, 16), (256, 1024, 16384, 10), (300, 256, 10000, 1), (256, 4096, 4736, 8),
+               (96, 200, 7000, 5), (256, 64, 18944, 10), (128, 512, 18945, 8), (255, 320, 2367, 10)]
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -245,10 +250,10 @@ def test_all_paths_agree_on_logits(vt):
     assert np.max(np.abs(a - b)) <= 2e-3 and np.max(np.abs(a - c)) <= 2e-3
 
 
-@pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (16, 1), (17, 2), (64, 2), (65, 2), (300, 4)])
+@pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (16, 1), (17, 2), (64, 2), (65, 2), (256, 2), (300, 3)])
 def test_launches_per_call_of_the_automatic_choice(vt, oracle, M, launches):
     # M = 1: GEMV; M <= 16: one launch, rows merged by the last warp to publish them; beyond: the same kernel in
-    # passes of 128 draft rows followed by the row-wise merge kernel
+    # passes of 256 draft rows (one tile per CTA, as here; 128 otherwise) followed by the row-wise merge kernel
     h, W, d2t = rand_case(M, 256, 3000, seed=40 + M)
     got = run_head(vt, h, dev_bf16(W), d2t, 4, vt.VT_PATH_AUTO)
     assert vt.vt_last_launch_count() == launches
