@@ -77,6 +77,7 @@ struct SmallParams {
     uint32_t w_tx;            // bytes one W box delivers (TH * 128)
     uint32_t h_blk;           // bytes of one k-block of h: 8 rows (M <= 8) or N rows x 128 B
     uint32_t h_off, lg_off, list_off, scratch_off, bar_off, total_smem;   // from the 1024-aligned base
+    uint32_t lg_bytes;        // one logits buffer (chunked thread-per-row has two, one per group of eight epilogue warps)
     uint32_t idesc;
 };
 
@@ -98,6 +99,7 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
 __device__ __forceinline__ void reader_barrier() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 // Barrier among the epilogue warps only (the producer and the MMA issuer never join it).
 __device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); }
+__device__ __forceinline__ void epi_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
 // KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue for more than 16 draft rows, with a
 // register list of KR >= k entries per thread.
@@ -328,8 +330,16 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         // different pipes (compare/select against multiply-add and exp2) and hide each other's latencies.
         constexpr int KL = KR > 0 ? KR : 1;
         // A CTA with a single tile takes its draft rows CH = 64 at a time and writes their records right away:
-        // shared memory then holds 64 rows of logits instead of all of them and the ring gets the difference.
-        const bool scanner = warp < 4;
+        // shared memory then holds 64 rows of logits per pass instead of all of them and the ring gets the
+        // difference.  Two groups of eight warps then work side by side, each with its own buffers and barrier,
+        // on every other pass: the scans wait on latencies more than on issue slots, so twice the warps finish
+        // in nearly half the time.
+        const int grp = warp >> 3, ngrp = p.n_epi >> 3;                // this warp's group; groups
+        const int wg = warp & 7;                                       // the warp within its group
+        const int gtid = tid & 255;
+        const int bar_id = 1 + 2 * grp;                                // named barriers 1 and 3 (2: the readers')
+        float* lg = reinterpret_cast<float*>(smem + p.lg_off + (uint32_t)grp * p.lg_bytes);
+        const bool scanner = wg < 4;
         const int w4 = warp & 3;
         const int CH = p.lg_rows;                                      // draft rows per pass of the epilogue
         const int nch = (M + CH - 1) / CH;                             // 1 unless the CTA has a single tile
@@ -358,16 +368,16 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (!got) fail();
                 }
             }
-            for (int ch = 0; ch < nch; ++ch) {
+            for (int ch = grp; ch < nch; ch += ngrp) {
                 const int m0 = ch * CH, Mc = min(CH, M - m0);          // this pass: draft rows m0 .. m0 + Mc - 1 of the launch
                 const float* rowp = lg + (size_t)min(m_own, Mc - 1) * kLgPitch;   // lanes past the last row re-read it and keep nothing
                 if (scanner) {
-                    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * p.N);
+                    const uint32_t taddr = tmem_base + ((uint32_t)(w4 * 32) << 16) + (uint32_t)(buf * p.N);
                     if (KF > 1) {
                         // Folded k-blocks (never with several passes): this warp's lanes are k-group g of tile rows
                         // r0 + lane, and columns NG*g .. NG*g + NG - 1 of the accumulator are their partial logits
                         // for the draft rows.
-                        const int SR = 128 / KF, NG = p.NG, g = (warp * 32) / SR, r = warp * 32 + lane - g * SR;
+                        const int SR = 128 / KF, NG = p.NG, g = (w4 * 32) / SR, r = w4 * 32 + lane - g * SR;
                         float* partial = reinterpret_cast<float*>(smem + p.part_off);
                         if (got) {
                             tc_fence_after();
@@ -383,7 +393,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                             if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
                         }
                         reader_barrier();                              // all four readers' partial sums are in place
-                        for (int e = tid; e < M * SR; e += 128) {
+                        for (int e = gtid; e < M * SR; e += 128) {
                             const int m = e / SR, rr = e - m * SR;
                             if (rr >= nv) continue;
                             float sum = 0.0f;
@@ -392,8 +402,8 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                             if (wants_logits(p.out)) store_logit(p.out, p.m_begin + m, row0 + rr, sum);
                         }
                     } else if (got) {
-                        const int i = warp * 32 + lane;                // TMEM lane = vocabulary row of the tile
-                        if (ch == 0) tc_fence_after();
+                        const int i = w4 * 32 + lane;                  // TMEM lane = vocabulary row of the tile
+                        if (ch == grp) tc_fence_after();
                         for (int c1 = 0; c1 < Mc; c1 += 16) {          // 16 draft rows per load
                             uint32_t u[16];
                             tc_ld16(taddr + (uint32_t)(m0 + c1), u);
@@ -410,24 +420,24 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                                 }
                             }
                         }
-                        if (ch == nch - 1) {                           // the accumulator is read out
+                        if (ch == nch - 1) {                           // the accumulator is read out (single-tile CTAs never wait for this)
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
                         }
                     }
                 }
-                epi_barrier(256);                                      // the pass's logits are in shared memory
+                epi_barrier(bar_id, 256);                                      // the pass's logits are in shared memory
                 // ---- the thread's own columns [cb, ce) of its draft row.  After a wait ran out the buffer holds
                 // older logits: whatever is computed from them belongs to a call that reports the time-out.
                 const int seg = (((nv + Q - 1) / Q) + 3) & ~3;         // multiples of 4: 16-byte loads
                 const int cb = part * seg, ce = min(nv, cb + seg), n = ce - cb;
                 if (works && n > 0 && !p.out.store_only) {
-                    if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + tid);
+                    if (scanner) row_scan_topk<KL>(rowp, cb, ce, row0, seen >= KL, v, ix, smem + p.scratch_off + (uint32_t)grp * (kRowQueue * 128) + gtid);
                     else row_scan_lse(rowp, cb, ce, mx, ssum);
                 }
                 seen += max(n, 0);
-                epi_barrier(256);                                      // the buffer may be overwritten
+                epi_barrier(bar_id, 256);                                      // the buffer may be overwritten
                 if (nch == 1 && t + 1 < ntiles) continue;              // lists and sums carry over to the next tile
                 // ---- the rows' records: best k keys and (max, sum-exp).  The logits buffer is free now: it takes
                 // every thread's list (or sums); the range-0 scanner of a row merges its column ranges and writes
@@ -441,7 +451,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         mine[KL] = pack_ms(mx, ssum);
                     }
                 }
-                epi_barrier(256);
+                epi_barrier(bar_id, 256);
                 if (scanner && part == 0 && m_own < Mc && !p.out.store_only) {
                     const int row = p.m_begin + m0 + m_own;                    // among the call's draft rows
                     // Q sorted lists: the best remaining key is the largest head, k times
@@ -469,14 +479,14 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     }
                     VT_ROW_MS(p.out, row)[cta] = pack_ms(cmx, cs);
                 }
-                if (ch + 1 < nch) {
-                    // the next pass starts from empty lists, once the exchange buffer has been read
+                if (ch + ngrp < nch) {
+                    // the group's next pass starts from empty lists, once the exchange buffer has been read
 #pragma unroll
                     for (int j = 0; j < KL; ++j) { v[j] = -INFINITY; ix[j] = -1; }
                     mx = -INFINITY;
                     ssum = 0.0f;
                     seen = 0;
-                    epi_barrier(256);
+                    epi_barrier(bar_id, 256);
                 }
             }
         }
@@ -660,13 +670,15 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, Sma
     const size_t lg_bytes = KR > 0 ? (std::max((size_t)p->lg_rows * kLgPitch * 4, (size_t)128 * (KR + 1) * 8) + 127) & ~(size_t)127
                                    : ((size_t)p->lg_rows * kLgPitch * 4 + 127) & ~(size_t)127;
     const size_t list_bytes = KR > 0 ? 0 : (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
-    p->n_epi = KR > 0 ? 8 : M > 8 ? kSmMaxEpiWarps : 8;
+    p->n_epi = KR > 0 ? (chunked ? 16 : 8) : M > 8 ? kSmMaxEpiWarps : 8;
     p->merge_in_kernel = KR == 0 && M <= p->n_epi;
     p->scratch_stride = (uint32_t)(kSmCand - VT_MAX_K + k) * 8u;
     // thread-per-row: the scanners' candidate queues, kRowQueue entries of one byte for each of 128 threads
-    const size_t scratch_bytes = KR > 0 ? (size_t)kRowQueue * 128 : ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
+    const size_t scratch_bytes = KR > 0 ? (size_t)kRowQueue * 128 * (chunked ? 2 : 1) : ((size_t)p->n_epi * p->scratch_stride + 127) & ~(size_t)127;
     const size_t bar_bytes = (size_t)(2 * kSmMaxStages + 4 + kHParts + 1) * 8 + 16;
-    const size_t common = 1024 + lg_bytes + list_bytes + scratch_bytes + bar_bytes + 128;
+    p->lg_bytes = (uint32_t)lg_bytes;
+    const size_t lg_total = lg_bytes * (chunked ? 2 : 1);
+    const size_t common = 1024 + lg_total + list_bytes + scratch_bytes + bar_bytes + 128;
     // h resident only for M <= 8 (8 rows per k-block) and short tiles, where little is streamed and the fold by two
     // wants it; otherwise it rides in the ring: measured 1-3 % faster at 109-row tiles once the ring (then six
     // stages instead of five) is filled ahead of the dependency wait.
@@ -712,7 +724,7 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, Sma
         p->h_off = (uint32_t)ring;                                            // stages are multiples of 1024 bytes
         p->part_off = (uint32_t)(ring + h_bytes);
         p->lg_off = (uint32_t)(p->part_off + part_bytes);
-        p->list_off = (uint32_t)(p->lg_off + lg_bytes);
+        p->list_off = (uint32_t)(p->lg_off + lg_total);
         p->scratch_off = (uint32_t)(p->list_off + list_bytes);
         p->bar_off = (uint32_t)(p->scratch_off + scratch_bytes);
         // An MMA always reads 128 A rows = 16 KB from its slot's first byte and N B rows from its h block's: past
