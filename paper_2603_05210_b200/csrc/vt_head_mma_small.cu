@@ -1,4 +1,4 @@
-// Draft head, tensor-core path with the vocabulary rows on the TMEM lanes (any M, 128 draft rows per launch).
+// Draft head, tensor-core path with the vocabulary rows on the TMEM lanes (any M, 128 or 256 draft rows per launch).
 //
 //   D[i, m] = sum_j W_trim[row0 + i, j] * h[m, j]       (the d -> k linear head, 2*d*k FLOPs per draft row)
 //
@@ -18,6 +18,10 @@
 //               ever waits for another.  With more rows a warp owns several, and merging them one after the other
 //               would put several round trips to L2 per row on the critical path: the kernel then only writes
 //               the records and a one-warp-per-row merge kernel follows it.
+//               From 17 draft rows on (from 9 or 13 when a CTA has a single tile, see small_plan) the epilogue is
+//               thread-per-row instead (KR > 0 below): warps 0-3 scan, warps 4-7 sum, records only; and with more
+//               than 64 draft rows on single-tile CTAs two such groups of eight warps take alternate passes of 64
+//               draft rows while pairs of CTAs share each MMA (PAIR below).
 //   next warp   TMA producer: boxes of 64 columns x tile-height rows of W (and the k-block of h) into a
 //               shared-memory ring
 //   last warp   MMA issuer: four K=16 tcgen05.mma (M=128, N) per 64-column k-block, tcgen05.commit frees the ring
@@ -101,8 +105,8 @@ __device__ __forceinline__ void reader_barrier() { asm volatile("bar.sync 2, 128
 __device__ __forceinline__ void epi_barrier(int threads) { asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory"); }
 __device__ __forceinline__ void epi_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
-// KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue for more than 16 draft rows, with a
-// register list of KR >= k entries per thread.
+// KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue (more than 16 draft rows, fewer on
+// single-tile CTAs), with a register list of KR >= k entries per thread.
 // PAIR: launched as clusters of two CTAs that share one MMA of 256 lanes (chunked thread-per-row only, one tile per
 // CTA): each CTA streams its own vocabulary rows and HALF of every k-block of h, so h crosses from L2 to the SMs
 // 74 times instead of 148 - with 128 and more draft rows that traffic, not the weight stream, was the bound.
@@ -648,8 +652,13 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, Sma
     const int nt = (R + 127) / 128;
     // More than 16 draft rows: one thread per draft row, as long as a register list holds k entries.  With four
     // and more tiles per CTA and at most 64 draft rows the warp-per-row epilogue hides behind the stream as well
-    // and leaves more shared memory to the ring (measured at V_trim = 128256: 180 against 194 us).
-    const int KR = (M > 16 && !(M <= 64 && nt >= 4)) ? topk_list_regs(k) : 0;
+    // and leaves more shared memory to the ring (measured at V_trim = 128256: 180 against 194 us).  With one tile
+    // per CTA nothing hides the epilogue, and thread-per-row is the faster one from 13 draft rows on, from 9 when
+    // k > 8 (measured at d = 4096, V_trim = 16384, k = 10: M = 16 37.3 -> 33.0 us, M = 9 36.0 -> 33.4 us; k = 8:
+    // M = 16 32.4 -> 31.5 us, M = 9..12 equal) although the rows are then merged by a second launch.
+    const bool many = M > 16 && !(M <= 64 && nt >= 4);
+    const bool few_single_tile = nt == 1 && (M > 12 || (M > 8 && k > 8));
+    const int KR = (many || few_single_tile) ? topk_list_regs(k) : 0;
     *list_regs = KR;
     // One tile per CTA and more than 64 draft rows: the epilogue takes the tile 64 draft rows at a time (nothing
     // carries over to a next tile), which frees 34 KB and more for the ring and lets one launch take 256 draft rows.

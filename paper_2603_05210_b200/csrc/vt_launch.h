@@ -75,9 +75,9 @@ inline cudaError_t launch_pdl_cluster2(void (*kernel)(KArgs...), int grid, int b
 bool gemv_supports(int d);
 vt_status launch_head_gemv(const HeadCall& c, cudaStream_t st, int* grid);
 vt_status launch_head_mma(const HeadCall& c, cudaStream_t st, int* grid);
-// any M, in passes of 128 draft rows; a single pass of at most 16 rows merges row by row in the same launch (one
-// arrival ticket per draft row), everything else launches the row-wise merge kernel after itself;
-// VT_ERR_UNSUPPORTED when the shape does not fit
+// any M, in passes of 128 draft rows (256 when every CTA has one tile of the vocabulary); a single pass of at most
+// 16 rows with the warp-per-row epilogue merges row by row in the same launch (one arrival ticket per draft row),
+// everything else launches the row-wise merge kernel after itself; VT_ERR_UNSUPPORTED when the shape does not fit
 vt_status launch_head_mma_small(const HeadCall& c, cudaStream_t st, int* grid);
 vt_status launch_merge_rowmajor(const HeadOut& o, int P, cudaStream_t st);   // one warp per draft row over the row-major records
 

@@ -172,7 +172,9 @@ HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8)
                # time, CTA pairs share each MMA, one launch holds up to 256 draft rows
                (65, 256, 5000, 10), (100, 1024, 16384, 10), (128, 512, 2368, 8), (129, 512, 18944, 4),
                (200, 2048, 9000, 16), (256, 1024, 16384, 10), (300, 256, 10000, 1), (256, 4096, 4736, 8),
-               (96, 200, 7000, 5), (256, 64, 18944, 10), (128, 512, 18945, 8), (255, 320, 2367, 10)]
+               (96, 200, 7000, 5), (256, 64, 18944, 10), (128, 512, 18945, 8), (255, 320, 2367, 10),
+               # 9 to 16 draft rows on single-tile CTAs: thread-per-row epilogue, with and without folded k-blocks
+               (16, 512, 3000, 10), (13, 256, 16384, 8), (10, 1024, 4096, 16), (16, 4096, 4096, 4), (9, 320, 9000, 9)]
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -250,10 +252,11 @@ def test_all_paths_agree_on_logits(vt):
     assert np.max(np.abs(a - b)) <= 2e-3 and np.max(np.abs(a - c)) <= 2e-3
 
 
-@pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (16, 1), (17, 2), (64, 2), (65, 2), (256, 2), (300, 3)])
+@pytest.mark.parametrize("M,launches", [(1, 1), (8, 1), (12, 1), (13, 2), (16, 2), (17, 2), (64, 2), (65, 2), (256, 2), (300, 3)])
 def test_launches_per_call_of_the_automatic_choice(vt, oracle, M, launches):
-    # M = 1: GEMV; M <= 16: one launch, rows merged by the last warp to publish them; beyond: the same kernel in
-    # passes of 256 draft rows (one tile per CTA, as here; 128 otherwise) followed by the row-wise merge kernel
+    # M = 1: GEMV; M <= 12 (16 with several tiles per CTA): one launch, rows merged by the last warp to publish them;
+    # beyond: the same kernel in passes of 256 draft rows (one tile per CTA, as here; 128 otherwise) followed by the
+    # row-wise merge kernel
     h, W, d2t = rand_case(M, 256, 3000, seed=40 + M)
     got = run_head(vt, h, dev_bf16(W), d2t, 4, vt.VT_PATH_AUTO)
     assert vt.vt_last_launch_count() == launches
