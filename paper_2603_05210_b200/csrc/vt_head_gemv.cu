@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
             ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
             if (ticket == (unsigned int)G - 1u) {
                 __threadfence();
-                merge_row_global(p.out, G, row);
+                merge_row_global(p.out, G, row, cbuf);
                 if (lane == 0) p.out.hdr->row_ticket[row] = 0u;        // ready for the next call
             }
         }

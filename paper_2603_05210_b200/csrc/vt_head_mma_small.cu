@@ -621,7 +621,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
             if (ticket == (unsigned int)G - 1u) {
                 __threadfence();
-                merge_row_global(p.out, G, row);
+                merge_row_global(p.out, G, row, cbuf);
                 if (lane == 0) p.out.hdr->row_ticket[row] = 0u;        // ready for the next call
             }
         }

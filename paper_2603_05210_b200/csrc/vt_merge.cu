@@ -11,7 +11,8 @@ constexpr int kMergeRowsPerCta = kMergeThreads / 32;
 __global__ void __launch_bounds__(kMergeThreads) merge_rowmajor_kernel(const HeadOut o, int P) {
     grid_dependency_wait();            // the head kernel's records must be complete
     const int m = blockIdx.x * kMergeRowsPerCta + (threadIdx.x >> 5);
-    if (m < o.M) merge_row_global(o, P, m);
+    __shared__ unsigned long long cbuf[kMergeRowsPerCta][kMergeCap];
+    if (m < o.M) merge_row_global(o, P, m, cbuf[threadIdx.x >> 5]);
 }
 
 vt_status launch_merge_rowmajor(const HeadOut& o, int P, cudaStream_t st) {

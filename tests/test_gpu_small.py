@@ -230,6 +230,26 @@ def test_exact_ties_resolve_to_lowest_draft_index(vt, oracle, path):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M,k", [(1, 8), (4, 10), (40, 8), (3, 16)])
+def test_all_winners_in_one_ctas_rows(vt, oracle, path, M, k):
+    # the k best logits of every draft row sit in adjacent vocabulary rows (one CTA's share): that CTA's list places
+    # more winners than the merge keeps in registers per list, the other lists none
+    rng = np.random.default_rng(50 + M + k)
+    d, Vt = 512, 6000
+    Wf = (0.02 * rng.standard_normal((Vt, d))).astype(np.float32)
+    hf = rng.standard_normal((M, d)).astype(np.float32)
+    hot = 1234 + np.arange(k + 3)
+    Wf[hot] = 0.05 * np.sign(hf.sum(axis=0))[None, :] * (1.0 + 0.01 * np.arange(k + 3))[:, None]   # same sign pattern as every row of h below
+    W = inputs.f32_to_bf16_bits(Wf).reshape(Vt, d)
+    h = inputs.f32_to_bf16_bits(np.abs(hf) * np.sign(hf.sum(axis=0))[None, :]).reshape(M, d)       # every row of h shares that sign pattern
+    d2t = np.arange(Vt, dtype=np.int32)[::-1].copy()
+    ora = oracle.draft_head(h, W, d2t, k, want_logits=True)
+    assert set(ora["draft_ids"][0].tolist()) <= set(hot.tolist())
+    got = run_head(vt, h, dev_bf16(W), d2t, k, path)
+    parity.check_head(got, ora, d2t, k)
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_same_input_twice_is_bit_identical_and_workspace_is_reusable(vt, oracle, path):
     h, W, d2t = rand_case(8, 1024, 5000, seed=9)
     Wd = dev_bf16(W)
