@@ -81,6 +81,7 @@ struct SmallParams {
     uint32_t w_tx;            // bytes one W box delivers (TH * 128)
     uint32_t h_blk;           // bytes of one k-block of h: 8 rows (M <= 8) or N rows x 128 B
     uint32_t h_off, lg_off, list_off, scratch_off, bar_off, total_smem;   // from the 1024-aligned base
+    int acce_count;           // arrivals that free an accumulator buffer: the reading warps of the CTA (of both CTAs of a pair)
     uint32_t lg_bytes;        // one logits buffer (chunked thread-per-row has two, one per group of eight epilogue warps)
     uint32_t idesc;
 };
@@ -107,8 +108,8 @@ __device__ __forceinline__ void epi_barrier(int id, int threads) { asm volatile(
 
 // KR == 0: the warp-per-row epilogue (any k).  KR > 0: the thread-per-row epilogue (more than 16 draft rows, fewer on
 // single-tile CTAs), with a register list of KR >= k entries per thread.
-// PAIR: launched as clusters of two CTAs that share one MMA of 256 lanes (chunked thread-per-row only, one tile per
-// CTA): each CTA streams its own vocabulary rows and HALF of every k-block of h, so h crosses from L2 to the SMs
+// PAIR: launched as clusters of two CTAs that share one MMA of 256 lanes (thread-per-row in passes of 64 draft rows
+// only): each CTA streams its own vocabulary rows and HALF of every k-block of h, so h crosses from L2 to the SMs
 // 74 times instead of 148 - with 128 and more draft rows that traffic, not the weight stream, was the bound.
 template <int KR, bool PAIR>
 __global__ void __launch_bounds__(kSmThreads, 1)
@@ -153,7 +154,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_accf + 8u * b, 1);
-            mbar_init(bar_acce + 8u * b, 4);
+            mbar_init(bar_acce + 8u * b, (uint32_t)p.acce_count);
         }
         for (int j = 0; j < kHParts; ++j) mbar_init(bar_h + 8u * j, 1);
         mbar_init(bar_drain, 1);
@@ -424,12 +425,31 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                                 }
                             }
                         }
-                        if (ch == nch - 1) {                           // the accumulator is read out (single-tile CTAs never wait for this)
+                        if (ch + ngrp >= nch) {                        // this group has read its share of the accumulator
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);   // the MMAs of the tile after next may start
+                            if (lane == 0) {                           // the MMAs of the tile after next may start
+                                if constexpr (PAIR) mbar_arrive_cluster(cluster_map_shared(bar_acce + 8u * buf, 0u));
+                                else mbar_arrive(bar_acce + 8u * buf);
+                            }
                         }
                     }
+                }
+                // A later tile of a CTA that works in passes: the rows' records so far (this CTA's own, from L2) join
+                // the merge below as one more list.  The summing threads fetch them now, under the scans.
+                constexpr int PV = (KL + 1) / 2;                       // keys of the old record per summing thread (Q = 2)
+                unsigned long long prevk[PV], prevms = 0ull;
+#pragma unroll
+                for (int i = 0; i < PV; ++i) prevk[i] = 0ull;
+                const bool carry = nch > 1 && t > 0;
+                if (carry && !scanner && works && m_own < Mc && !p.out.store_only) {
+                    const int row = p.m_begin + m0 + m_own;
+#pragma unroll
+                    for (int i = 0; i < PV; ++i) {
+                        const int j = part + Q * i;
+                        prevk[i] = j < k ? __ldcg(VT_ROW_KEYS(p.out, row, j) + cta) : 0ull;
+                    }
+                    if (part == 0) prevms = __ldcg(VT_ROW_MS(p.out, row) + cta);
                 }
                 epi_barrier(bar_id, 256);                                      // the pass's logits are in shared memory
                 // ---- the thread's own columns [cb, ce) of its draft row.  After a wait ran out the buffer holds
@@ -453,19 +473,27 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         for (int j = 0; j < KL; ++j) mine[j] = ix[j] >= 0 ? make_key(v[j], ix[j]) : 0ull;
                     } else {
                         mine[KL] = pack_ms(mx, ssum);
+                        if (carry && m_own < Mc) {                             // list Q: the record of the earlier tiles
+                            unsigned long long* old = xl + (size_t)(Q * xs + m_own) * (KL + 1);
+#pragma unroll
+                            for (int i = 0; i < PV; ++i)
+                                if (part + Q * i < KL) old[part + Q * i] = prevk[i];
+                            if (part == 0) old[KL] = prevms;
+                        }
                     }
                 }
                 epi_barrier(bar_id, 256);
+                const int NL = Q + (carry ? 1 : 0);                            // sorted lists per row
                 if (scanner && part == 0 && m_own < Mc && !p.out.store_only) {
                     const int row = p.m_begin + m0 + m_own;                    // among the call's draft rows
-                    // Q sorted lists: the best remaining key is the largest head, k times
+                    // NL sorted lists: the best remaining key is the largest head, k times
                     int pos[4] = {0, 0, 0, 0};
                     for (int j = 0; j < k; ++j) {
                         unsigned long long best = 0ull;
                         int bq = 0;
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            if (q < Q && pos[q] < KL) {
+                            if (q < NL && pos[q] < KL) {
                                 const unsigned long long key = xl[(size_t)(q * xs + m_own) * (KL + 1) + pos[q]];
                                 if (key > best) { best = key; bq = q; }
                             }
@@ -475,15 +503,15 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         VT_ROW_KEYS(p.out, row, j)[cta] = best;
                     }
                     float cmx = -INFINITY;
-                    for (int q = 0; q < Q; ++q) cmx = fmaxf(cmx, unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]).x);
+                    for (int q = 0; q < NL; ++q) cmx = fmaxf(cmx, unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]).x);
                     float cs = 0.0f;
-                    for (int q = 0; q < Q; ++q) {
+                    for (int q = 0; q < NL; ++q) {
                         const float2 ms = unpack_ms(xl[(size_t)(q * xs + m_own) * (KL + 1) + KL]);
                         if (ms.y > 0.0f) cs += ms.y * __expf(ms.x - cmx);
                     }
                     VT_ROW_MS(p.out, row)[cta] = pack_ms(cmx, cs);
                 }
-                if (ch + ngrp < nch) {
+                if (ch + ngrp < nch || t + 1 < ntiles) {
                     // the group's next pass starts from empty lists, once the exchange buffer has been read
 #pragma unroll
                     for (int j = 0; j < KL; ++j) { v[j] = -INFINITY; ix[j] = -1; }
@@ -660,9 +688,13 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, Sma
     const bool few_single_tile = nt == 1 && (M > 12 || (M > 8 && k > 8));
     const int KR = (many || few_single_tile) ? topk_list_regs(k) : 0;
     *list_regs = KR;
-    // One tile per CTA and more than 64 draft rows: the epilogue takes the tile 64 draft rows at a time (nothing
-    // carries over to a next tile), which frees 34 KB and more for the ring and lets one launch take 256 draft rows.
-    const bool chunked = KR > 0 && nt == 1 && M > kChunkRows;
+    // More than 64 draft rows: the epilogue takes a tile 64 draft rows at a time and writes (from the second tile on:
+    // merges into) their records at once, so nothing but the records carries over between passes; that halves the
+    // logits buffer at 128 draft rows and lets one launch take 256.
+    // With several tiles per CTA and at most 96 draft rows one pass per tile with the lists kept in registers is as
+    // good or better (measured at V_trim = 128256, M = 65: 181 against 202 us; M = 100: equal; V_trim = 32000, M = 100:
+    // 72 against 64 us).
+    const bool chunked = KR > 0 && M > kChunkRows && (nt == 1 || M > 96);
     if (M > kSmMaxM && !chunked) return false;
     // ... and then two CTAs share each MMA, each fetching half of h
     const bool pair = chunked && pairs_ok && (grid & 1) == 0;
@@ -680,6 +712,7 @@ static bool small_plan(int M, int d, int Vt, int k, int grid, bool pairs_ok, Sma
                                    : ((size_t)p->lg_rows * kLgPitch * 4 + 127) & ~(size_t)127;
     const size_t list_bytes = KR > 0 ? 0 : (((size_t)M * k * 8 + (size_t)kSmMaxM * 12) + 127) & ~(size_t)127;
     p->n_epi = KR > 0 ? (chunked ? 16 : 8) : M > 8 ? kSmMaxEpiWarps : 8;
+    p->acce_count = chunked ? (pair ? 16 : 8) : 4;
     p->merge_in_kernel = KR == 0 && M <= p->n_epi;
     p->scratch_stride = (uint32_t)(kSmCand - VT_MAX_K + k) * 8u;
     // thread-per-row: the scanners' candidate queues, kRowQueue entries of one byte for each of 128 threads

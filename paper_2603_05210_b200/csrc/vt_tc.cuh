@@ -66,6 +66,10 @@ __device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t r
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// One arrival on an mbarrier of another CTA of the cluster (`bar_cluster` from cluster_map_shared).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
 // TMA box into this CTA's shared memory, completion bytes on `bar_cluster` (a shared::cluster address: rank 0's barrier).
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
     asm volatile(

@@ -173,6 +173,9 @@ HEAD_SHAPES = [(1, 64, 1, 1), (1, 64, 7, 7), (1, 2048, 4380, 1), (3, 64, 127, 8)
                (65, 256, 5000, 10), (100, 1024, 16384, 10), (128, 512, 2368, 8), (129, 512, 18944, 4),
                (200, 2048, 9000, 16), (256, 1024, 16384, 10), (300, 256, 10000, 1), (256, 4096, 4736, 8),
                (96, 200, 7000, 5), (256, 64, 18944, 10), (128, 512, 18945, 8), (255, 320, 2367, 10),
+               # ... and with several tiles per CTA: the rows' records carry over between the tiles (two tiles; three and
+               # four, where the MMA issuer waits for both CTAs' readers before it reuses an accumulator buffer)
+               (256, 256, 40000, 10), (200, 512, 60000, 4), (65, 128, 20000, 16), (130, 320, 75000, 8),
                # 9 to 16 draft rows on single-tile CTAs: thread-per-row epilogue, with and without folded k-blocks
                (16, 512, 3000, 10), (13, 256, 16384, 8), (10, 1024, 4096, 16), (16, 4096, 4096, 4), (9, 320, 9000, 9)]
 
