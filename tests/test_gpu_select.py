@@ -41,6 +41,15 @@ def test_small_streams(vt, V, N, seed):
     check(vt, tokens, V, 64, 5e4, 0.5, 0.0, max(1, V // 3), max(1, V // 2))
 
 
+def test_coverage_exactly_at_the_threshold_is_admitted(vt):
+    # Eq. 5: C(k) >= c_min keeps U(k); counts 5, 3, 2 give C(2) = 8/10 = the double 0.8
+    tokens = np.array([0] * 5 + [1] * 3 + [2] * 2, dtype=np.int32)
+    got, _ = check(vt, tokens, 3, 4, 10.0, 0.2, 0.8, 1, 3)
+    assert got["k_star"] == 2
+    got, _ = check(vt, tokens, 3, 4, 10.0, 0.2, float(np.nextafter(0.8, 1.0)), 1, 3)
+    assert got["k_star"] == 3
+
+
 def test_llama3_vocabulary_paper_constants(vt):
     V = inputs.V_LLAMA3
     tokens = inputs.zipf_token_stream(V, 1.1, 1_000_000, seed=11)

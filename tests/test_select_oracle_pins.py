@@ -127,3 +127,15 @@ def test_unique_coverage_vs_set_arithmetic_and_table4_shape():
     C = so.coverage_curve(f, order)
     uc = so.unique_coverage_curve(f, order)
     assert C[13263] > 0.85 and uc[13263] < 0.5 * C[13263]                  # frequent ids carry the mass; most distinct ids are rare
+
+
+def test_coverage_exactly_at_the_threshold_is_admitted():
+    # Eq. 5 keeps U(k) when C(k) >= c_min: counts 5, 3, 2 give C = 0.5, 0.8, 1.0 and 8/10 is the double 0.8, so with
+    # c_min = 0.8 and a utility that falls with k the answer is k = 2 (k = 1 is penalised, k = 3 scores less)
+    tok = np.array([0] * 5 + [1] * 3 + [2] * 2, dtype=np.int32)
+    r = so.select(tok, V=3, d=4, F_fixed=10.0, alpha=0.2, c_min=0.8, k_min=1, k_max=3)
+    assert list(r["C"]) == [0.5, 0.8, 1.0]
+    assert r["U_pen"][0] == -1.0 and r["U_pen"][1] == r["U"][1] and r["U"][1] > r["U"][2]
+    assert r["k_star"] == 2 and r["C_star"] == 0.8
+    # a hair above the threshold value excludes it
+    assert so.select(tok, V=3, d=4, F_fixed=10.0, alpha=0.2, c_min=np.nextafter(0.8, 1.0), k_min=1, k_max=3)["k_star"] == 3
