@@ -241,8 +241,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) head_gemv_kernel(const GemvPa
         // CTAs) merges the row at once, straight from global memory, with no CTA-wide step between the fold and
         // the outputs.  With many draft rows the row-wise merge kernel follows instead.
         const int row = p.m_begin + m;
-        warp_select_topk(rec0, stride, P1, k, cbuf,
-                         [&](int j, unsigned long long best) { VT_ROW_KEYS(p.out, row, j)[cta] = best; });
+        auto to_record = [&](int j, unsigned long long best) { VT_ROW_KEYS(p.out, row, j)[cta] = best; };
+        if (P1 <= 32 && k <= kSelectLanesMaxK) warp_select_topk_lanes(rec0, stride, P1, k, cbuf, to_record);
+        else warp_select_topk(rec0, stride, P1, k, cbuf, to_record);
         if (lane == 0) VT_ROW_MS(p.out, row)[cta] = pack_ms(ms.x, ms.y);
         if (p.out.fused_merge) {
             __threadfence();
