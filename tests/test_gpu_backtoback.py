@@ -31,7 +31,7 @@ def vt():
     return vt
 
 
-def make_sets(M, seed):
+def make_sets(M, seed, D=D, VT=VT):
     """Three (h, W_trim, d2t) sets that give three different answers."""
     sets = []
     for s in range(3):
@@ -86,6 +86,33 @@ def test_unsynchronised_calls_on_a_shared_workspace_match_the_oracle(vt, oracle,
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             enqueue_all(vt, dev_sets, outs, ws, static_weights)
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    graph.replay()
+    assert vt.vt_last_status(ws) == vt.VT_OK
+    check_all(outs, refs, sets, M)
+
+
+@pytest.mark.parametrize("M", [130, 256])
+def test_unsynchronised_calls_many_rows_several_tiles_per_cta(vt, oracle, M):
+    # CTA pairs sharing each MMA, passes of 64 draft rows, three tiles per CTA: the rows' records carry over between
+    # tiles through the workspace the calls share, and the MMA issuer waits for both CTAs' readers
+    sets = make_sets(M, 9300 + M, D=256, VT=40000)
+    refs = [oracle.draft_head(h, W, d2t, K, want_logits=True) for h, W, d2t in sets]
+    dev_sets = [(dev_bf16(h), dev_bf16(W), dev_i32(d2t)) for h, W, d2t in sets]
+    ws = vt.new_workspace(vt.vt_workspace_bytes(M, K))
+    outs = fresh_outs(M)
+    torch.cuda.synchronize()
+    enqueue_all(vt, dev_sets, outs, ws, False)
+    assert vt.vt_last_status(ws) == vt.VT_OK
+    check_all(outs, refs, sets, M)
+    outs = fresh_outs(M)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            enqueue_all(vt, dev_sets, outs, ws, False)
     torch.cuda.current_stream().wait_stream(side)
     graph.replay()
     graph.replay()
