@@ -44,112 +44,169 @@ __global__ void __launch_bounds__(512) select_hist_kernel(const int32_t* __restr
 }
 
 // ------------------------------------------------------------------------------------------ sort
-// Stable LSD radix sort of V (key, id) pairs by one CTA of 1024 threads, 8 bits per pass.
-// key = key_max - count, so ascending keys are descending counts; ids start ascending and every pass is
-// stable, so equal counts stay in ascending id order.
+// Stable LSD radix sort of V (key, id) pairs, 8 bits per pass, over kSortBlocks CTAs that each own one contiguous
+// chunk of the array: per pass every CTA counts its chunk's digits, one CTA turns the counts into output positions
+// (digit-major, CTA-minor: all of digit 0 first, within a digit the chunks in order), and every CTA scatters its
+// chunk in order.  key = key_max - count, so ascending keys are descending counts; ids start ascending and every
+// pass is stable, so equal counts stay in ascending id order.
 constexpr int kSortThreads = 1024;
+constexpr int kSortBlocks = 128;
 
-__global__ void __launch_bounds__(kSortThreads) select_sort_kernel(const unsigned int* __restrict__ counts, int V,
-                                                                    unsigned int key_max, int passes,
-                                                                    unsigned int* keyA, int* valA,
-                                                                    unsigned int* keyB, int* valB) {
-    __shared__ unsigned int base[256];                 // running output position of each digit
-    __shared__ unsigned int warp_cnt[32][256];         // per chunk: occurrences of each digit in each warp
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    for (int i = tid; i < V; i += kSortThreads) {
+__host__ __device__ inline int sort_chunk(int V) {            // elements per CTA: whole sub-chunks of kSortThreads
+    const int per = (V + kSortBlocks - 1) / kSortBlocks;
+    return ((per + kSortThreads - 1) / kSortThreads) * kSortThreads;
+}
+
+__global__ void __launch_bounds__(kSortThreads) select_keys_kernel(const unsigned int* __restrict__ counts, int V,
+                                                                    unsigned int key_max, unsigned int* keyA, int* valA) {
+    for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < V; i += gridDim.x * kSortThreads) {
         keyA[i] = key_max - counts[i];
         valA[i] = i;
     }
+}
+
+__global__ void __launch_bounds__(kSortThreads) sort_count_kernel(const unsigned int* __restrict__ kin, int V, int shift,
+                                                                   unsigned int* __restrict__ hist) {
+    __shared__ unsigned int cnt[256];
+    const int tid = threadIdx.x;
+    if (tid < 256) cnt[tid] = 0;
     __syncthreads();
-    unsigned int* kin = keyA;
-    unsigned int* kout = keyB;
-    int* vin = valA;
-    int* vout = valB;
-    for (int pass = 0; pass < passes; ++pass) {
-        const int shift = 8 * pass;
-        if (tid < 256) base[tid] = 0;
-        __syncthreads();
-        for (int i = tid; i < V; i += kSortThreads) atomicAdd(&base[(kin[i] >> shift) & 255u], 1u);
-        __syncthreads();
-        if (warp == 0) {                                // exclusive scan of the 256 digit counts
-            unsigned int run = 0;
-            for (int c = 0; c < 8; ++c) {
-                const unsigned int v = base[c * 32 + lane];
-                unsigned int inc = v;
+    const int chunk = sort_chunk(V), begin = blockIdx.x * chunk, end = min(V, begin + chunk);
+    for (int i = begin + tid; i < end; i += kSortThreads) atomicAdd(&cnt[(kin[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    if (tid < 256) hist[tid * kSortBlocks + blockIdx.x] = cnt[tid];
+}
+
+// Exclusive prefix sum of the 256 x kSortBlocks counts in place (one CTA; 32 consecutive entries per thread).
+__global__ void __launch_bounds__(kSortThreads) sort_offsets_kernel(unsigned int* __restrict__ hist) {
+    __shared__ unsigned int warp_tot[32];
+    constexpr int PER = 256 * kSortBlocks / kSortThreads;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    unsigned int v[PER], sum = 0;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= o) inc += n;
-                }
-                base[c * 32 + lane] = run + inc - v;
-                run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+    for (int j = 0; j < PER; ++j) { v[j] = hist[tid * PER + j]; sum += v[j]; }
+    unsigned int inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    unsigned int run = inc - sum;
+    for (int w = 0; w < warp; ++w) run += warp_tot[w];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) { hist[tid * PER + j] = run; run += v[j]; }
+}
+
+__global__ void __launch_bounds__(kSortThreads) sort_scatter_kernel(const unsigned int* __restrict__ kin,
+                                                                     const int* __restrict__ vin, int V, int shift,
+                                                                     const unsigned int* __restrict__ offs,
+                                                                     unsigned int* __restrict__ kout, int* __restrict__ vout) {
+    __shared__ unsigned int base[256];                 // running output position of each digit for this CTA's chunk
+    __shared__ unsigned int warp_cnt[32][256];         // per sub-chunk: occurrences of each digit in each warp
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid < 256) base[tid] = offs[tid * kSortBlocks + blockIdx.x];
+    __syncthreads();
+    const int chunk = sort_chunk(V), begin = blockIdx.x * chunk, end = min(V, begin + chunk);
+    for (int c0 = begin; c0 < end; c0 += kSortThreads) {
+        const int i = c0 + tid;
+        const bool ok = i < end;
+        const unsigned int key = ok ? kin[i] : 0u;
+        const int val = ok ? vin[i] : 0;
+        const unsigned int dg = ok ? (key >> shift) & 255u : 256u;     // 256: a lane past the end
+        for (int j = lane; j < 256; j += 32) warp_cnt[warp][j] = 0;
+        __syncwarp();
+        const unsigned int peers = __match_any_sync(0xFFFFFFFFu, dg);
+        const unsigned int before = __popc(peers & ((1u << lane) - 1u));
+        if (ok && before == 0) warp_cnt[warp][dg] = __popc(peers);
+        __syncthreads();
+        if (tid < 256) {                                // digit tid: warps in order, then advance its base
+            unsigned int run = base[tid];
+            for (int w = 0; w < 32; ++w) {
+                const unsigned int n = warp_cnt[w][tid];
+                warp_cnt[w][tid] = run;
+                run += n;
             }
+            base[tid] = run;
         }
         __syncthreads();
-        for (int c0 = 0; c0 < V; c0 += kSortThreads) {
-            const int i = c0 + tid;
-            const bool ok = i < V;
-            const unsigned int key = ok ? kin[i] : 0u;
-            const int val = ok ? vin[i] : 0;
-            const unsigned int dg = ok ? (key >> shift) & 255u : 256u;     // 256: a lane past the end
-            for (int j = lane; j < 256; j += 32) warp_cnt[warp][j] = 0;
-            __syncwarp();
-            const unsigned int peers = __match_any_sync(0xFFFFFFFFu, dg);
-            const unsigned int before = __popc(peers & ((1u << lane) - 1u));
-            if (ok && before == 0) warp_cnt[warp][dg] = __popc(peers);
-            __syncthreads();
-            if (tid < 256) {                            // digit tid: warps in order, then advance its base
-                unsigned int run = base[tid];
-                for (int w = 0; w < 32; ++w) {
-                    const unsigned int n = warp_cnt[w][tid];
-                    warp_cnt[w][tid] = run;
-                    run += n;
-                }
-                base[tid] = run;
-            }
-            __syncthreads();
-            if (ok) {
-                const unsigned int pos = warp_cnt[warp][dg] + before;
-                kout[pos] = key;
-                vout[pos] = val;
-            }
-            __syncthreads();
+        if (ok) {
+            const unsigned int pos = warp_cnt[warp][dg] + before;
+            kout[pos] = key;
+            vout[pos] = val;
         }
-        unsigned int* tk = kin; kin = kout; kout = tk;
-        int* tv = vin; vin = vout; vout = tv;
-    }
-    // an odd number of passes leaves the result in the B buffers: bring it back to A
-    if (kin != keyA) {
-        for (int i = tid; i < V; i += kSortThreads) {
-            keyA[i] = kin[i];
-            valA[i] = vin[i];
-        }
+        __syncthreads();
     }
 }
 
 // ------------------------------------------------------------------------------------------ scan + objective
-__global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* __restrict__ key_sorted,
-                                                           const int* __restrict__ val_sorted, int V,
-                                                           unsigned int key_max, int d, double F_fixed, double alpha,
-                                                           double c_min, int k_min, int k_max,
-                                                           unsigned long long* __restrict__ cum,
-                                                           int32_t* __restrict__ ranked_ids,
-                                                           unsigned long long* __restrict__ cum_out,
-                                                           SelectResult* result) {
+// Over the same kSortBlocks chunks: (1) every CTA sums its chunk's counts and counts the ids that occur;
+// (2) every CTA adds the sums of the chunks before it, scans its chunk, writes the cumulative counts and the ranking,
+// and evaluates the objective for the k of its chunk; (3) one small CTA picks the best of the CTAs' bests.
+struct ScanScratch {
+    unsigned long long sum[kSortBlocks];
+    double best_u[kSortBlocks], best_c[kSortBlocks], best_r[kSortBlocks];
+    int best_k[kSortBlocks];
+    unsigned int distinct[kSortBlocks];
+};
+
+__global__ void __launch_bounds__(kSortThreads) scan_sums_kernel(const unsigned int* __restrict__ key_sorted, int V,
+                                                                  unsigned int key_max, ScanScratch* sc) {
+    __shared__ unsigned long long wsum[32];
+    __shared__ unsigned int wocc[32];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk = sort_chunk(V), begin = blockIdx.x * chunk, end = min(V, begin + chunk);
+    unsigned long long s = 0ull;
+    unsigned int occ = 0u;
+    for (int i = begin + tid; i < end; i += kSortThreads) {
+        const unsigned int v = key_max - key_sorted[i];
+        s += v;
+        occ += v > 0u ? 1u : 0u;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        occ += __shfl_xor_sync(0xFFFFFFFFu, occ, o);
+    }
+    if (lane == 0) { wsum[warp] = s; wocc[warp] = occ; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 32; ++w) { s += wsum[w]; occ += wocc[w]; }
+        sc->sum[blockIdx.x] = s;
+        sc->distinct[blockIdx.x] = occ;
+    }
+}
+
+__global__ void __launch_bounds__(kSortThreads) scan_apply_kernel(const unsigned int* __restrict__ key_sorted,
+                                                                   const int* __restrict__ val_sorted, int V,
+                                                                   unsigned int key_max, int d, double F_fixed, double alpha,
+                                                                   double c_min, int k_min, int k_max,
+                                                                   unsigned long long* __restrict__ cum,
+                                                                   int32_t* __restrict__ ranked_ids,
+                                                                   unsigned long long* __restrict__ cum_out,
+                                                                   ScanScratch* sc) {
     __shared__ unsigned long long warp_tot[32];
-    __shared__ unsigned long long carry_s;
-    __shared__ unsigned int distinct_s;      // ids that occur at all (count > 0): they sort first
-    __shared__ double best_u[32];
+    __shared__ unsigned long long carry_s, total_s;
+    __shared__ double best_u[32], best_c[32], best_r[32];
     __shared__ int best_k[32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) { carry_s = 0ull; distinct_s = 0u; }
+    const int chunk = sort_chunk(V), begin = blockIdx.x * chunk, end = min(V, begin + chunk);
+    if (tid == 0) {
+        unsigned long long before = 0ull, all = 0ull;
+        for (int b = 0; b < kSortBlocks; ++b) {
+            const unsigned long long s = sc->sum[b];
+            if (b < (int)blockIdx.x) before += s;
+            all += s;
+        }
+        carry_s = before;
+        total_s = all;
+    }
     __syncthreads();
-    for (int c0 = 0; c0 < V; c0 += 1024) {              // inclusive prefix sum of the sorted counts
+    for (int c0 = begin; c0 < end; c0 += kSortThreads) {   // inclusive prefix sum of the sorted counts
         const int i = c0 + tid;
-        unsigned long long v = i < V ? (unsigned long long)(key_max - key_sorted[i]) : 0ull;
-        if (i < V) ranked_ids[i] = val_sorted[i];
-        const unsigned int occurs = __ballot_sync(0xFFFFFFFFu, v > 0ull);
-        if (lane == 0 && occurs) atomicAdd(&distinct_s, (unsigned int)__popc(occurs));
+        unsigned long long v = i < end ? (unsigned long long)(key_max - key_sorted[i]) : 0ull;
+        if (i < end) ranked_ids[i] = val_sorted[i];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const unsigned long long n = __shfl_up_sync(0xFFFFFFFFu, v, o);
@@ -160,15 +217,15 @@ __global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* _
         unsigned long long off = carry_s;
         for (int w = 0; w < warp; ++w) off += warp_tot[w];
         v += off;
-        if (i < V) {
+        if (i < end) {
             cum[i] = v;
             if (cum_out) cum_out[i] = v;
         }
         __syncthreads();
-        if (tid == 1023) carry_s = v;
+        if (tid == kSortThreads - 1) carry_s = v;
         __syncthreads();
     }
-    const unsigned long long total = carry_s;
+    const unsigned long long total = total_s;
     const double tot_d = (double)total;
     const double two_d = __dmul_rn(2.0, (double)d);
     const double denom = __dadd_rn(F_fixed, __dmul_rn(two_d, (double)V));
@@ -176,8 +233,11 @@ __global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* _
     double bu = -2.0, bc = 0.0, br = 0.0;
     int bk = 0x7FFFFFFF;
     if (total > 0) {
-        for (int k = k_min + tid; k <= k_max; k += 1024) {    // each thread meets its k in ascending order
-            const double C = __ddiv_rn((double)cum[k - 1], tot_d);
+        // k = i + 1 for the chunk's positions i; every thread reads back what it wrote itself
+        for (int i = begin + tid; i < end; i += kSortThreads) {
+            const int k = i + 1;
+            if (k < k_min || k > k_max) continue;
+            const double C = __ddiv_rn((double)cum[i], tot_d);
             const double R = __dsub_rn(1.0, __ddiv_rn(__dadd_rn(F_fixed, __dmul_rn(two_d, (double)k)), denom));
             const double U = __dadd_rn(__dmul_rn(alpha, C), __dmul_rn(one_minus_alpha, R));
             const double Up = C >= c_min ? U : -1.0;
@@ -193,25 +253,44 @@ __global__ void __launch_bounds__(1024) select_scan_kernel(const unsigned int* _
         const double orr = __shfl_xor_sync(0xFFFFFFFFu, br, o);
         if (ou > bu || (ou == bu && ok < bk)) { bu = ou; bk = ok; bc = oc; br = orr; }
     }
-    __shared__ double best_c[32], best_r[32];
     if (lane == 0) { best_u[warp] = bu; best_k[warp] = bk; best_c[warp] = bc; best_r[warp] = br; }
     __syncthreads();
     if (tid == 0) {
         for (int w = 1; w < 32; ++w)
             if (best_u[w] > bu || (best_u[w] == bu && best_k[w] < bk)) { bu = best_u[w]; bk = best_k[w]; bc = best_c[w]; br = best_r[w]; }
-        result->k_star = total > 0 ? bk : 0;
-        result->C = bc;
-        result->R = br;
-        result->U = bu;
-        result->total = total;
-        // counts descend, so the ids that occur are exactly the first distinct_s of the ranking (Table 4's
-        // "unique coverage": kept distinct ids over all distinct ids)
-        const unsigned int distinct = distinct_s;
-        result->unique = distinct > 0 ? __ddiv_rn((double)min((unsigned int)max(bk, 0), distinct), (double)distinct) : 0.0;
+        sc->best_u[blockIdx.x] = bu;
+        sc->best_k[blockIdx.x] = bk;
+        sc->best_c[blockIdx.x] = bc;
+        sc->best_r[blockIdx.x] = br;
     }
 }
 
+__global__ void __launch_bounds__(32) scan_pick_kernel(const ScanScratch* sc, SelectResult* result) {
+    if (threadIdx.x != 0) return;
+    double bu = -2.0, bc = 0.0, br = 0.0;
+    int bk = 0x7FFFFFFF;
+    unsigned long long total = 0ull;
+    unsigned int distinct = 0u;
+    for (int b = 0; b < kSortBlocks; ++b) {
+        total += sc->sum[b];
+        distinct += sc->distinct[b];
+        if (sc->best_u[b] > bu || (sc->best_u[b] == bu && sc->best_k[b] < bk)) {
+            bu = sc->best_u[b]; bk = sc->best_k[b]; bc = sc->best_c[b]; br = sc->best_r[b];
+        }
+    }
+    result->k_star = total > 0 ? bk : 0;
+    result->C = bc;
+    result->R = br;
+    result->U = bu;
+    result->total = total;
+    // counts descend, so the ids that occur are exactly the first `distinct` of the ranking (Table 4's
+    // "unique coverage": kept distinct ids over all distinct ids)
+    result->unique = distinct > 0 ? __ddiv_rn((double)min((unsigned int)max(bk, 0), distinct), (double)distinct) : 0.0;
+}
+
 static inline size_t up256s(size_t b) { return (b + 255) & ~(size_t)255; }
+constexpr size_t kSortHistBytes = (size_t)256 * kSortBlocks * 4;
+constexpr size_t kSelectScratchBytes = kSortHistBytes + ((sizeof(ScanScratch) + 255) & ~(size_t)255);
 
 }  // namespace vt
 
@@ -220,7 +299,8 @@ using namespace vt;
 extern "C" size_t vt_select_workspace_bytes(int V_full) {
     if (V_full < 1) return 0;
     const size_t v = (size_t)V_full;
-    return 256 + up256s(v * 4) * 5 + up256s(v * 8);     // result | counts | keyA keyB valA valB | cum
+    // result | counts | keyA keyB valA valB | cum | digit counts of the sort | partial sums of the scan
+    return 256 + up256s(v * 4) * 5 + up256s(v * 8) + kSelectScratchBytes;
 }
 
 extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_full, int d, double F_fixed, double alpha,
@@ -249,6 +329,7 @@ extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_
     int* valA = reinterpret_cast<int*>(base + 256 + 3 * a4);
     int* valB = reinterpret_cast<int*>(base + 256 + 4 * a4);
     unsigned long long* cum = reinterpret_cast<unsigned long long*>(base + 256 + 5 * a4);
+    unsigned int* hist = reinterpret_cast<unsigned int*>(base + 256 + 5 * a4 + up256s((size_t)V_full * 8));
 
     cudaError_t e = cudaMemsetAsync(base, 0, 256 + a4, st);          // result and counts
     if (e != cudaSuccess) return cuda_fail(e);
@@ -263,10 +344,27 @@ extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_
     while (bits < 32 && (1ll << bits) <= N) ++bits;
     const unsigned int key_max = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
     const int passes = (bits + 7) / 8;
-    select_sort_kernel<<<1, kSortThreads, 0, st>>>(counts, V_full, key_max, passes, keyA, valA, keyB, valB);
+    select_keys_kernel<<<std::min(kSortBlocks, (V_full + kSortThreads - 1) / kSortThreads), kSortThreads, 0, st>>>(counts, V_full, key_max, keyA, valA);
     count_launch();
-    select_scan_kernel<<<1, 1024, 0, st>>>(keyA, valA, V_full, key_max, d, F_fixed, alpha, c_min, k_min, k_max, cum,
-                                           ranked_ids, reinterpret_cast<unsigned long long*>(cum_counts), result);
+    unsigned int *kin = keyA, *kout = keyB;
+    int *vin = valA, *vout = valB;
+    for (int pass = 0; pass < passes; ++pass) {
+        sort_count_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, V_full, 8 * pass, hist);
+        sort_offsets_kernel<<<1, kSortThreads, 0, st>>>(hist);
+        sort_scatter_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, vin, V_full, 8 * pass, hist, kout, vout);
+        count_launch();
+        count_launch();
+        count_launch();
+        std::swap(kin, kout);
+        std::swap(vin, vout);
+    }
+    ScanScratch* sc = reinterpret_cast<ScanScratch*>(reinterpret_cast<unsigned char*>(hist) + kSortHistBytes);
+    scan_sums_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, V_full, key_max, sc);
+    scan_apply_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, vin, V_full, key_max, d, F_fixed, alpha, c_min, k_min, k_max, cum,
+                                                            ranked_ids, reinterpret_cast<unsigned long long*>(cum_counts), sc);
+    scan_pick_kernel<<<1, 32, 0, st>>>(sc, result);
+    count_launch();
+    count_launch();
     count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e);
