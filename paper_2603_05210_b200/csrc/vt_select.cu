@@ -8,10 +8,10 @@
 //   k*     = argmax over k in [k_min, k_max] of U~(k), smallest k among equal maxima    (Eq. 1)
 //
 // The paper samples 100 values of k with a TPE optimiser; evaluating every k costs one pass over a
-// 128K-entry prefix sum, so the scan returns the exact optimum of the same objective.  Three kernels:
+// 128K-entry prefix sum, so the scan returns the exact optimum of the same objective.  Three steps:
 // a histogram with warp-aggregated atomics (HBM-bound read of the stream), a stable least-significant-
-// digit radix sort of (count, id) in one CTA (the vocabulary is only ~128K entries), and a scan +
-// objective + arg-max kernel in one CTA.  Doubles are combined with explicit round-to-nearest
+// digit radix sort of (count, id), and a prefix sum + objective + arg-max, the last two over 128 CTAs
+// that each own one contiguous chunk of the vocabulary.  Doubles are combined with explicit round-to-nearest
 // operations so that no fused multiply-add changes a result against the fp64 definition.
 #include "vt_launch.h"
 
