@@ -77,26 +77,35 @@ __global__ void __launch_bounds__(kSortThreads) sort_count_kernel(const unsigned
     if (tid < 256) hist[tid * kSortBlocks + blockIdx.x] = cnt[tid];
 }
 
-// Exclusive prefix sum of the 256 x kSortBlocks counts in place (one CTA; 32 consecutive entries per thread).
+// Exclusive prefix sum of the 256 x kSortBlocks counts in place (one CTA).  Warp w owns the 1024 consecutive
+// entries from 1024 w: it loads them as 32 coalesced rows of 32, scans row after row with a running carry, and adds
+// the totals of the warps before it.
 __global__ void __launch_bounds__(kSortThreads) sort_offsets_kernel(unsigned int* __restrict__ hist) {
+    static_assert(256 * kSortBlocks == 32 * kSortThreads, "one 1024-entry segment per warp");
     __shared__ unsigned int warp_tot[32];
-    constexpr int PER = 256 * kSortBlocks / kSortThreads;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    unsigned int v[PER], sum = 0;
+    unsigned int* seg = hist + warp * 1024;
+    unsigned int v[32];
 #pragma unroll
-    for (int j = 0; j < PER; ++j) { v[j] = hist[tid * PER + j]; sum += v[j]; }
-    unsigned int inc = sum;
+    for (int j = 0; j < 32; ++j) v[j] = seg[j * 32 + lane];
+    unsigned int carry = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += n;
+    for (int j = 0; j < 32; ++j) {
+        unsigned int inc = v[j];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += n;
+        }
+        v[j] = carry + inc - v[j];                       // exclusive, within the segment
+        carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
     }
-    if (lane == 31) warp_tot[warp] = inc;
+    if (lane == 0) warp_tot[warp] = carry;
     __syncthreads();
-    unsigned int run = inc - sum;
-    for (int w = 0; w < warp; ++w) run += warp_tot[w];
+    unsigned int before = 0;
+    for (int w = 0; w < warp; ++w) before += warp_tot[w];
 #pragma unroll
-    for (int j = 0; j < PER; ++j) { hist[tid * PER + j] = run; run += v[j]; }
+    for (int j = 0; j < 32; ++j) seg[j * 32 + lane] = before + v[j];
 }
 
 __global__ void __launch_bounds__(kSortThreads) sort_scatter_kernel(const unsigned int* __restrict__ kin,
@@ -265,18 +274,24 @@ __global__ void __launch_bounds__(kSortThreads) scan_apply_kernel(const unsigned
     }
 }
 
-__global__ void __launch_bounds__(32) scan_pick_kernel(const ScanScratch* sc, SelectResult* result) {
-    if (threadIdx.x != 0) return;
+__global__ void __launch_bounds__(kSortBlocks) scan_pick_kernel(const ScanScratch* sc, SelectResult* result) {
+    __shared__ unsigned long long s_sum[kSortBlocks];
+    __shared__ unsigned int s_dis[kSortBlocks];
+    __shared__ double s_u[kSortBlocks], s_c[kSortBlocks], s_r[kSortBlocks];
+    __shared__ int s_k[kSortBlocks];
+    const int b = threadIdx.x;
+    s_sum[b] = sc->sum[b]; s_dis[b] = sc->distinct[b];
+    s_u[b] = sc->best_u[b]; s_k[b] = sc->best_k[b]; s_c[b] = sc->best_c[b]; s_r[b] = sc->best_r[b];
+    __syncthreads();
+    if (b != 0) return;
     double bu = -2.0, bc = 0.0, br = 0.0;
     int bk = 0x7FFFFFFF;
     unsigned long long total = 0ull;
     unsigned int distinct = 0u;
-    for (int b = 0; b < kSortBlocks; ++b) {
-        total += sc->sum[b];
-        distinct += sc->distinct[b];
-        if (sc->best_u[b] > bu || (sc->best_u[b] == bu && sc->best_k[b] < bk)) {
-            bu = sc->best_u[b]; bk = sc->best_k[b]; bc = sc->best_c[b]; br = sc->best_r[b];
-        }
+    for (int i = 0; i < kSortBlocks; ++i) {
+        total += s_sum[i];
+        distinct += s_dis[i];
+        if (s_u[i] > bu || (s_u[i] == bu && s_k[i] < bk)) { bu = s_u[i]; bk = s_k[i]; bc = s_c[i]; br = s_r[i]; }
     }
     result->k_star = total > 0 ? bk : 0;
     result->C = bc;
@@ -362,7 +377,7 @@ extern "C" vt_status vt_select_vocab(const int32_t* token_ids, int64_t N, int V_
     scan_sums_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, V_full, key_max, sc);
     scan_apply_kernel<<<kSortBlocks, kSortThreads, 0, st>>>(kin, vin, V_full, key_max, d, F_fixed, alpha, c_min, k_min, k_max, cum,
                                                             ranked_ids, reinterpret_cast<unsigned long long*>(cum_counts), sc);
-    scan_pick_kernel<<<1, 32, 0, st>>>(sc, result);
+    scan_pick_kernel<<<1, kSortBlocks, 0, st>>>(sc, result);
     count_launch();
     count_launch();
     count_launch();
