@@ -50,7 +50,8 @@ typedef enum vt_path {
     VT_PATH_GEMV = 1,      /* CUDA-core streaming GEMV; 4 draft rows per pass, d <= 8192              */
     VT_PATH_MMA = 2,       /* tcgen05 tensor-core GEMM, draft rows on the TMEM lanes; any M            */
     VT_PATH_MMA_SMALL = 3  /* tcgen05 tensor-core GEMM, vocabulary rows on the TMEM lanes; any M, in passes
-                              of 128 draft rows                                                        */
+                              of 128 draft rows; of 256 when k <= 16 and M > 96 (M > 64 where a CTA owns at
+                              most 128 vocabulary rows): pairs of CTAs then share each MMA            */
 } vt_path;
 
 #define VT_PATH_MASK 0xFF  /* the vt_path part of an `options` argument */
