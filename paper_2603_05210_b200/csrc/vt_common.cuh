@@ -421,9 +421,10 @@ __device__ __forceinline__ float warp_topk_update(const float* vals, int ncols, 
         if (is_cand) cbuf[n + __popc(m & ((1u << lane) - 1u))] = make_key(v[i], col0 + lane + 32 * i);
         n += __popc(m);
     }
-    for (int j = lane; j < k; j += 32) cbuf[n + j] = list[j];      // empty slots are 0 and rank last
+    const int kl = list[0] != 0ull ? k : 0;                       // an empty list (the row's first tile) has nothing to rank
+    for (int j = lane; j < kl; j += 32) cbuf[n + j] = list[j];     // empty slots are 0 and rank last
     __syncwarp();
-    const int total = n + k;
+    const int total = n + kl;
     for (int e = lane; e < total; e += 32) {
         const unsigned long long key = cbuf[e];
         int rank = 0;
