@@ -399,7 +399,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         }
                         reader_barrier();                              // all four readers' partial sums are in place
                         for (int e = gtid; e < M * SR; e += 128) {
-                            const int m = e / SR, rr = e - m * SR;
+                            const int m = e >> (KF == 4 ? 5 : 6), rr = e & (SR - 1);            // SR = 128 / KF is 32 or 64
                             if (rr >= nv) continue;
                             float sum = 0.0f;
                             for (int gg = 0; gg < KF; ++gg) sum += partial[(gg * p.NG + m) * 64 + rr];
@@ -580,7 +580,7 @@ head_mma_small_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     }
                     reader_barrier();                                  // all four readers' partial sums are in place
                     for (int e = tid; e < M * SR; e += 128) {
-                        const int m = e / SR, rr = e - m * SR;
+                        const int m = e >> (KF == 4 ? 5 : 6), rr = e & (SR - 1);            // SR = 128 / KF is 32 or 64
                         if (rr >= nv) continue;
                         float sum = 0.0f;
                         for (int gg = 0; gg < KF; ++gg) sum += part[(gg * p.NG + m) * 64 + rr];
