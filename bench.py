@@ -48,7 +48,7 @@ def head_bytes(d, Vt, M, k):
 # DRAM traffic of one head launch on the bench workload from the ncu capture summarised in
 # profiles/head_mma_small_d4096_vt32000_m8.md (dram__bytes_read.sum + dram__bytes_write.sum), valid while the
 # kernel sources still hash to the value recorded there.
-NCU_TRAFFIC = {"bytes": 264_385_792 + 3_609_344, "source_hash": "4346eada1892888c",
+NCU_TRAFFIC = {"bytes": 264_363_520 + 4_110_080, "source_hash": "ac01381d7e9f9884",
                "sources": ("paper_2603_05210_b200/csrc/vt_head_mma_small.cu", "paper_2603_05210_b200/csrc/vt_common.cuh",
                            "paper_2603_05210_b200/csrc/vt_tc.cuh")}
 
